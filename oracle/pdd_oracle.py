@@ -208,35 +208,45 @@ def refine_topk(score, kind, cand_lo: int, cand_hi: int, keep_ratio: float):
     return keep, int(keep.sum()), k
 
 
-def sentence_values(score, kind, seg_start, dtype=np.float64):
+def sentence_values(score, kind, seg_start):
     """Value of each sentence = mean score of its prompt tokens (Sec. 3.2: the KVCache of one
     sentence is treated as a whole).  The aggregator is not given in the paper; the mean is
-    this build's reading ("parity unpinned").  Returns (value [n_seg], count [n_seg]); a
-    sentence without prompt tokens has count 0 and value -inf.
-
-    dtype=float32 repeats the kernel's arithmetic for the decision (tokens added one by one
-    in position order, then one division), dtype=float64 is the plain definition."""
-    score = np.asarray(score)
+    this build's reading ("parity unpinned").  Returns (value [n_seg] fp64, count [n_seg]); a
+    sentence without prompt tokens has count 0 and value -inf."""
+    score = np.asarray(score, dtype=np.float64)
     n_seg = len(seg_start) - 1
     kind = np.zeros(len(score), np.uint8) if kind is None else np.asarray(kind, np.uint8)
-    value = np.full(n_seg, -np.inf, dtype=dtype)
+    value = np.full(n_seg, -np.inf, dtype=np.float64)
     count = np.zeros(n_seg, dtype=np.int64)
     for s in range(n_seg):
-        acc = dtype(0)
-        c = 0
-        for i in range(int(seg_start[s]), int(seg_start[s + 1])):
-            if kind[i] == PROMPT:
-                acc = dtype(acc + dtype(score[i]))
-                c += 1
-        count[s] = c
-        if c:
-            value[s] = dtype(acc / dtype(c))
+        sl = slice(int(seg_start[s]), int(seg_start[s + 1]))
+        prompt = kind[sl] == PROMPT
+        count[s] = int(prompt.sum())
+        if count[s]:
+            value[s] = math.fsum(score[sl][prompt]) / float(count[s])
     return value, count
 
 
-def refine_sentences(score, kind, seg_start, keep_ratio: float, dtype=np.float64):
-    """Sentence-level selection (Sec. 3.2: "the selection of KVCache implies the selection of
-    sentences"; Sec. 4, Table 2: the "Refine (Sentences)" variant).
+def select_sentences(value, count, budget: int) -> np.ndarray:
+    """Which sentences are taken, given their values, their prompt-token counts and the token
+    budget: sentences are visited by decreasing value (ties: lower sentence first) and one is
+    taken iff it has prompt tokens and still fits what is left of the budget."""
+    value = np.asarray(value, dtype=np.float64)
+    order = np.argsort(-value, kind="stable")
+    taken = np.zeros(len(value), dtype=bool)
+    rem = int(budget)
+    for s in order:
+        if rem == 0:
+            break
+        if 0 < count[s] <= rem:
+            taken[s] = True
+            rem -= int(count[s])
+    return taken
+
+
+def refine_sentences(score, kind, seg_start, keep_ratio: float):
+    """Sentence-level selection (Sec. 3.2: choosing KVCache entries amounts to choosing whole
+    sentences; Sec. 4, Table 2: the "Refine (Sentences)" variant).
 
     seg_start [n_seg+1] are sentence boundaries that tile the content range
     [seg_start[0], seg_start[-1]); prompt positions outside it (prefix, suffix) are always kept,
@@ -244,7 +254,7 @@ def refine_sentences(score, kind, seg_start, keep_ratio: float, dtype=np.float64
     #content prompt tokens), sentences are visited by decreasing value (ties: lower sentence
     first) and a sentence is taken iff it still fits the remaining budget, until the budget
     is used up.  Returns (keep uint8 [n], n_kept, taken [n_seg] bool)."""
-    score = np.asarray(score)
+    score = np.asarray(score, dtype=np.float64)
     n = len(score)
     kind = np.zeros(n, np.uint8) if kind is None else np.asarray(kind, np.uint8)
     seg_start = np.asarray(seg_start, dtype=np.int64)
@@ -255,16 +265,8 @@ def refine_sentences(score, kind, seg_start, keep_ratio: float, dtype=np.float64
     always = is_prompt & ~content
     k_total = keep_count(keep_ratio, int(is_prompt.sum()))
     budget = min(max(k_total - int(always.sum()), 0), int(content.sum()))
-    value, count = sentence_values(score, kind, seg_start, dtype)
-    order = np.argsort(-value.astype(np.float64), kind="stable")
-    taken = np.zeros(len(value), dtype=bool)
-    rem = budget
-    for s in order:
-        if rem == 0:
-            break
-        if 0 < count[s] <= rem:
-            taken[s] = True
-            rem -= int(count[s])
+    value, count = sentence_values(score, kind, seg_start)
+    taken = select_sentences(value, count, budget)
     keep = np.zeros(n, dtype=np.uint8)
     keep[always] = 1
     for s in np.nonzero(taken)[0]:
@@ -281,51 +283,25 @@ def pack_mask_bits(keep) -> np.ndarray:
     return np.packbits(keep != 0, bitorder="little")
 
 
-def pool1d_as(x, kind: str, width: int, dtype):
-    """pool1d in a chosen precision: dtype=float64 is pool1d itself; dtype=float32 repeats a
-    single-precision evaluation (window entries added one by one from the lowest position,
-    one division by the width) so that a decision taken on fp32 values can be replayed."""
-    x = np.asarray(x, dtype=dtype)
-    if kind == "none" or width == 1:
-        return x.copy()
-    assert width % 2 == 1 and width >= 1
-    half = width // 2
-    n = x.shape[-1]
-    out = np.empty_like(x)
-    for j in range(n):
-        lo, hi = max(0, j - half), min(n, j + half + 1)
-        if kind == "avg":
-            acc = np.zeros(x.shape[:-1], dtype=dtype)
-            for t in range(lo, hi):
-                acc = (acc + x[..., t]).astype(dtype)
-            out[..., j] = (acc / dtype(width)).astype(dtype)
-        elif kind == "max":
-            out[..., j] = x[..., lo:hi].max(axis=-1)
-        else:
-            raise ValueError(kind)
-    return out
-
-
 def refine_vote(colsum, kind, cand_lo: int, cand_hi: int, keep_ratio: float,
-                pool_kind: str = "none", pool_width: int = 1, dtype=np.float64):
-    """Per-head selection followed by a vote (Sec. 3.2: "we select the indices with top values
-    (with ratio r) per head", yet ONE mask of the prompt's length is sent).  The paper does not
-    say how the per-head index sets become one mask; this is the alternative to summing the
-    heads first ("parity unpinned" as a reading):
+                pool_kind: str = "none", pool_width: int = 1):
+    """Per-head selection followed by a vote (Sec. 3.2 picks the top-valued indices of every
+    head at ratio r, yet ONE mask of the prompt's length is sent).  The paper does not say how
+    the per-head index sets become one mask; this is the alternative to summing the heads first
+    ("parity unpinned" as a reading):
 
       1. every head h selects its own k candidates with the largest pooled column sums
          (the same candidates, the same k and the same tie rule as refine_topk);
       2. votes[j] = number of heads that selected position j;
       3. the mask keeps the k candidates with the most votes; equal votes are ordered by the
-         summed pooled column sums (heads added in index order), then by the lower position.
+         pooled column sums added over the heads, then by the lower position.
 
-    colsum is [n_heads, n].  dtype selects the precision in which pooled values and the head
-    sum are formed (float32 replays a single-precision evaluation for the integer decision).
-    Returns (keep uint8 [n], n_kept, votes int32 [n])."""
-    cs = np.asarray(colsum)
+    colsum is [n_heads, n].  Returns (keep uint8 [n], n_kept, votes int32 [n], total fp64 [n])
+    with total the head sum of the pooled values."""
+    cs = np.asarray(colsum, dtype=np.float64)
     n_heads, n = cs.shape
     kind = np.zeros(n, dtype=np.uint8) if kind is None else np.asarray(kind, dtype=np.uint8)
-    pooled = pool1d_as(cs, pool_kind, pool_width, dtype)
+    pooled = pool1d(cs, pool_kind, pool_width)
     pos = np.arange(n)
     is_prompt = kind == PROMPT
     cand = is_prompt & (pos >= cand_lo) & (pos < cand_hi)
@@ -335,16 +311,14 @@ def refine_vote(colsum, kind, cand_lo: int, cand_hi: int, keep_ratio: float,
     for h in range(n_heads):
         keep_h, _, k = refine_topk(pooled[h], kind, cand_lo, cand_hi, keep_ratio)
         votes += (keep_h.astype(bool) & cand).astype(np.int32)
-    total = np.zeros(n, dtype=dtype)
-    for h in range(n_heads):
-        total = (total + pooled[h]).astype(dtype)
+    total = pooled.sum(axis=0)
     idx = pos[cand]
     # descending votes, then descending total, then ascending position
-    order = np.lexsort((idx, -total[idx].astype(np.float64), -votes[idx]))
+    order = np.lexsort((idx, -total[idx], -votes[idx]))
     keep = np.zeros(n, dtype=np.uint8)
     keep[always] = 1
     keep[idx[order[:k]]] = 1
-    return keep, int(keep.sum()), votes
+    return keep, int(keep.sum()), votes, total
 
 
 def solve_rl(l: float, k_c: float, k_d: float, delta: float, delta_c: float, xi: float,

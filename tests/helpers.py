@@ -194,3 +194,95 @@ def compare_full(w: wl.Workload, got, want, cand=None, what: str = ""):
         np.testing.assert_array_equal(got[si]["keep"], own, err_msg=tag + " mask vs own scores")
         stats.append(dict(out_max=mx, out_mean=mean, imp_rel=rel, band=band, keep_diff=diff))
     return stats
+
+
+# ---------------------------------------------------------------------------------------------
+# Single-precision replays.  SECONDARY checks only: the parity statements of the sentence and
+# vote selections are made against the fp64 checker (bands below); these functions repeat an
+# fp32 evaluation (terms added one by one in position / head order, one division) so that a
+# test can also say "and the mask is the exact selection for the values the library formed".
+
+def replay_sentence_values_f32(score, kind, seg_start):
+    score = np.asarray(score, dtype=np.float32)
+    n_seg = len(seg_start) - 1
+    kind = np.zeros(len(score), np.uint8) if kind is None else np.asarray(kind, np.uint8)
+    value = np.full(n_seg, -np.inf, dtype=np.float32)
+    count = np.zeros(n_seg, dtype=np.int64)
+    for s in range(n_seg):
+        acc = np.float32(0)
+        c = 0
+        for i in range(int(seg_start[s]), int(seg_start[s + 1])):
+            if kind[i] == wl.PROMPT:
+                acc = np.float32(acc + score[i])
+                c += 1
+        count[s] = c
+        if c:
+            value[s] = np.float32(acc / np.float32(c))
+    return value, count
+
+
+def replay_pool_f32(x, kind: str, width: int):
+    x = np.asarray(x, dtype=np.float32)
+    if kind == "none" or width == 1:
+        return x.copy()
+    half = width // 2
+    n = x.shape[-1]
+    out = np.empty_like(x)
+    for j in range(n):
+        lo, hi = max(0, j - half), min(n, j + half + 1)
+        if kind == "avg":
+            acc = np.zeros(x.shape[:-1], dtype=np.float32)
+            for t in range(lo, hi):
+                acc = (acc + x[..., t]).astype(np.float32)
+            out[..., j] = (acc / np.float32(width)).astype(np.float32)
+        else:
+            out[..., j] = x[..., lo:hi].max(axis=-1)
+    return out
+
+
+def sentence_budget(kind, seg_start, keep_ratio: float) -> int:
+    """Token budget of the sentence selection: clamp(k_total - #always_kept, 0, #content)."""
+    from oracle import pdd_oracle as orc
+    n = len(kind)
+    pos = np.arange(n)
+    prompt = np.asarray(kind) == wl.PROMPT
+    content = prompt & (pos >= int(seg_start[0])) & (pos < int(seg_start[-1]))
+    always = prompt & ~content
+    k_total = orc.keep_count(keep_ratio, int(prompt.sum()))
+    return min(max(k_total - int(always.sum()), 0), int(content.sum()))
+
+
+def sentence_near_ties(value64, count, rel: float) -> int:
+    """Adjacent pairs (in decreasing order) of distinct sentence values closer than rel: the
+    pairs whose order an fp32 evaluation of the means may turn round."""
+    v = np.sort(np.asarray(value64)[np.asarray(count) > 0])[::-1]
+    if len(v) < 2:
+        return 0
+    gap = v[:-1] - v[1:]
+    return int(((gap > 0) & (gap <= rel * np.abs(v[:-1]))).sum())
+
+
+def check_vote_keep(keep_gpu, n_kept_gpu, votes_gpu, keep_o, n_kept_o, votes_o, total_o, kind,
+                    cand_lo: int, cand_hi: int, n_heads: int, what: str = ""):
+    """Vote selection against the fp64 checker.  Votes must agree exactly (the caller only
+    passes inputs whose per-head decisions are exact in fp32).  The mask must agree outside the
+    near-tie band: candidates with the threshold's vote count whose head sum lies within the
+    fp32 summation error of the threshold's head sum.  Returns the band size."""
+    np.testing.assert_array_equal(votes_gpu, votes_o, err_msg=what + " votes")
+    assert n_kept_gpu == n_kept_o == int(keep_gpu.sum()), what + " popcount"
+    n = len(keep_o)
+    pos = np.arange(n)
+    cand = (np.asarray(kind) == wl.PROMPT) & (pos >= cand_lo) & (pos < cand_hi)
+    k = int(keep_o[cand].sum())
+    band = np.zeros(n, dtype=bool)
+    if 0 < k < int(cand.sum()):
+        idx = pos[cand]
+        order = np.lexsort((idx, -total_o[idx], -votes_o[idx]))
+        last = idx[order[k - 1]]
+        v_star, theta = votes_o[last], total_o[last]
+        eps = (n_heads + 2) * 2.0 ** -24 * np.abs(total_o)
+        band = cand & (votes_o == v_star) & (np.abs(total_o - theta) <= 2 * (eps + eps[last]))
+    mism = int((keep_gpu[~band] != keep_o[~band]).sum())
+    assert mism == 0, "%s: %d mask mismatches outside the near-tie band (band %d)" % (
+        what, mism, int(band.sum()))
+    return int(band.sum())

@@ -1,6 +1,9 @@
 """GPU parity of per-head selection with a vote (index work: the bar is bit-exact).  The
-library and the checker get the same fp32 column sums; pooled values and the head sum are
-formed in fp32 on both sides, so every decision is taken in the same precision."""
+library pools and adds heads in fp32; the checker is the fp64 definition.  The inputs are
+chosen so that every per-head decision is exact in fp32 (no pooling, max pooling, or
+average pooling of multiples of 1/8), hence the vote counts must agree exactly; the head sum
+that orders equal vote counts carries fp32 rounding, so the mask must agree outside the
+near-tie band around the threshold's head sum and have the same popcount."""
 import numpy as np
 import pytest
 
@@ -35,7 +38,7 @@ def _run_vote(cs, kind, lo, hi, ratio, pool, width, ld_pad=0):
 
 
 @pytest.mark.parametrize("n,heads", [(9, 3), (300, 8), (4160, 32), (33024, 32), (5000, 70)])
-def test_vote_matches_checker(n, heads):
+def test_vote_matches_fp64_checker(n, heads):
     from oracle import pdd_oracle as orc
     rng = wl.rng_for(600 + n + heads)
     cases = [(0.0, "none", 1), (0.3, "none", 1), (0.5, "max", 3), (1.0, "none", 1)]
@@ -45,21 +48,23 @@ def test_vote_matches_checker(n, heads):
         # heavy-tailed column sums, heads that agree on some positions and differ on others
         shared = rng.random(n) ** 6
         cs = (0.5 * shared[None, :] + rng.random((heads, n)) ** 4).astype(np.float32)
-        if ratio == 0.5:
-            cs = (np.round(cs * 8) / 8).astype(np.float32)             # many exact ties
+        if ratio == 0.5 or pool == "avg":
+            cs = (np.round(cs * 8) / 8).astype(np.float32)   # exact ties; exact fp32 window sums
         kind = (rng.random(n) < 0.05).astype(np.uint8)
         lo, hi = int(rng.integers(0, n // 10 + 1)), n - int(rng.integers(0, n // 10 + 1))
         keep, n_kept, votes = _run_vote(cs, kind, lo, hi, ratio, pool, width, ld_pad=int(n % 7))
-        want, want_n, want_votes = orc.refine_vote(cs, kind, lo, hi, ratio, pool, width,
-                                                   dtype=np.float32)
-        np.testing.assert_array_equal(votes, want_votes)
-        np.testing.assert_array_equal(keep, want)
-        assert n_kept == want_n
+        want, want_n, want_votes, total = orc.refine_vote(cs, kind, lo, hi, ratio, pool, width)
+        band = H.check_vote_keep(keep, n_kept, votes, want, want_n, want_votes, total, kind, lo,
+                                 hi, heads, "vote n=%d heads=%d r=%g %s" % (n, heads, ratio, pool))
+        assert band <= max(8, n // 50), "near-tie band of %d positions: the check is vacuous" % band
+        if pool != "avg":
+            # multiples of 1/8 add exactly in fp32 too: there the mask is the checker's, bit for bit
+            if ratio == 0.5:
+                np.testing.assert_array_equal(keep, want)
 
 
 def test_vote_on_library_column_sums():
-    """End of the path: column sums from the attention pass, exported, then the vote.  With one
-    head group the vote and the sum-first rule are both valid masks of the same size."""
+    """End of the path: column sums from the attention pass, exported, then the vote."""
     import torch
     from oracle import pdd_oracle as orc
     w = wl.small_like("vote", 610, 8, 2, 128, 900, 256, 20, keep_ratio=0.3, window="last")
@@ -71,10 +76,11 @@ def test_vote_on_library_column_sums():
         fn(H.to_dev(s.q[sl]), H.to_dev(s.k[sl]), H.to_dev(s.v[sl]), window=c.window)
     cs = kv.export_colsum(0).cpu().numpy()
     keep, n_kept, votes = _run_vote(cs, s.kind, 16, 880, 0.3, "none", 1)
-    want, want_n, want_votes = orc.refine_vote(cs, s.kind, 16, 880, 0.3, dtype=np.float32)
-    np.testing.assert_array_equal(keep, want)
-    np.testing.assert_array_equal(votes, want_votes)
-    assert n_kept == want_n == orc.keep_count(0.3, s.n_prompt)
+    want, want_n, want_votes, total = orc.refine_vote(cs, s.kind, 16, 880, 0.3)
+    band = H.check_vote_keep(keep, n_kept, votes, want, want_n, want_votes, total, s.kind, 16,
+                             880, 8, "vote on library column sums")
+    assert band <= 8
+    assert n_kept == orc.keep_count(0.3, s.n_prompt)
     assert not keep[s.kind == 1].any()
     kv.close()
 

@@ -67,7 +67,7 @@ def test_sentence_selection_invariants():
             assert not taken.any()
 
 
-def test_sentence_value_is_the_mean_of_prompt_tokens_and_f32_mode_is_sequential():
+def test_sentence_value_is_the_mean_of_prompt_tokens():
     score = np.array([1.0, 2.0, 6.0, 10.0, 3.0, 5.0])
     kind = np.array([0, 0, 1, 0, 0, 0], np.uint8)
     v, c = orc.sentence_values(score, kind, [0, 3, 4, 6])
@@ -75,12 +75,19 @@ def test_sentence_value_is_the_mean_of_prompt_tokens_and_f32_mode_is_sequential(
     assert list(c) == [2, 1, 2]
     v, c = orc.sentence_values(score, np.array([1, 1, 1, 0, 0, 0], np.uint8), [0, 3, 6])
     assert v[0] == -np.inf and c[0] == 0 and abs(v[1] - 6.0) < 1e-15
-    # float32 mode adds one by one in float32 (a sum the fp64 mean would not reproduce)
+    # fp32 inputs are widened before they are added (a single-precision sum would lose the ones)
     s32 = np.array([1e8, 1.0, 1.0, 1.0, 1.0], np.float32)
-    v32, _ = orc.sentence_values(s32, None, [0, 5], dtype=np.float32)
-    assert v32[0] == np.float32(np.float32(1e8) / np.float32(5))
     v64, _ = orc.sentence_values(s32, None, [0, 5])
     assert v64[0] == (1e8 + 4) / 5
+
+
+def test_select_sentences_is_first_fit_by_decreasing_value():
+    value = np.array([0.5, 0.9, 0.9, -np.inf, 0.1])
+    count = np.array([3, 4, 2, 0, 1])
+    # order 1, 2, 0, 4: 4 tokens, then 2 (fits 6), then 3 does not fit the 1 left, then 1 fits
+    assert list(orc.select_sentences(value, count, 7)) == [False, True, True, False, True]
+    assert list(orc.select_sentences(value, count, 3)) == [False, False, True, False, True]
+    assert not orc.select_sentences(value, count, 0).any()
 
 
 def test_golden_sentence_example():
