@@ -10,6 +10,20 @@
  * nothing throws, aborts or traps.  Device-side problems (a bounded wait that ran out)
  * set a sticky word that pdd_status reads.
  *
+ * One stream per handle.  Every call on a pdd_kv shares the handle's scratch (row
+ * normalisers, partial results of split key ranges, the ring of call records, cached tensor
+ * maps) without any synchronisation of its own: issue all calls of a handle on ONE stream,
+ * or order them with events so that the kernels of two calls never overlap on the GPU.
+ * Handles are independent of one another.  The host part of a handle is not thread-safe.
+ *
+ * After a failure.  A hot call that returns an error before or while it enqueues its kernels
+ * leaves the handle's host state (lengths, pages) as it found it, so the same call can be
+ * repeated; cache rows a partly enqueued call may have written lie beyond the sequences'
+ * lengths and are overwritten by the next call at those positions.  Once the sticky word is
+ * PDD_ERR_TIMEOUT, every later kernel of the handle returns without doing any work (outputs
+ * are not written) until pdd_clear_status; what the interrupted kernels left in the cache is
+ * undefined, so reset the sequences that were in flight (pdd_kv_reset) before reusing them.
+ *
  * Conventions
  *   q, out : bf16, token-major [rows][n_q_heads][head_dim], contiguous, 16-byte aligned
  *   k, v   : bf16, token-major [rows][n_kv_heads][head_dim], contiguous, 16-byte aligned
@@ -73,9 +87,9 @@ typedef struct {
 } pdd_batch;
 
 /*
- * KV cache set-up.  "All necessary intermediate data is stored in HBM (e.g. KVCache)"
- * and grows with the prompt (Sec. 2.1 and Sec. 3.2, preliminaries): the cache is a pool
- * of fixed-size pages plus a page table per sequence.
+ * KV cache set-up.  The KV cache and the other intermediate data stay in HBM and grow with
+ * the prompt (Sec. 2.1 and Sec. 3.2, preliminaries): the cache is a pool of fixed-size pages
+ * plus a page table per sequence.
  *
  * pdd_kv_bytes_required: size of the device arena for a configuration.
  * pdd_kv_alloc: dev_buf is device memory of at least that size, 256-byte aligned, owned
@@ -170,22 +184,25 @@ int pdd_refine_topk_batched(const float* score, const uint8_t* kinds, int32_t n_
  *   keep      : uint8 [n]; n_kept: int32 on the device (<= floor(keep_ratio*l + 1/2)).
  *   seg_value : optional fp32 [n_seg] (device) receiving the sentence values, or NULL.
  * 1 <= n_seg <= 8192 (PDD_ERR_CAPACITY beyond); score, kinds as in pdd_refine_topk.
+ * seg_start is device memory, so the host cannot validate it: the kernel checks that every
+ * boundary lies in [0, n] and that they do not decrease.  If they do not, nothing is read or
+ * written through a bad boundary: keep is all zeros and n_kept is -1.
  */
 int pdd_refine_sentences(const float* score, const uint8_t* kinds, int64_t n,
                          const int32_t* seg_start, int32_t n_seg, double keep_ratio,
                          uint8_t* keep, int32_t* n_kept, float* seg_value, void* stream);
 
 /*
- * pdd_pack_mask -- the mask tensor as a bit stream (Sec. 3.2: "we further treat it as a bit
- * stream" before compression): bit (i mod 8) of bits[i / 8] = (keep[i] != 0), least
+ * pdd_pack_mask -- the mask tensor as a bit stream (Sec. 3.2 serialises the mask as a bit
+ * stream before it is compressed): bit (i mod 8) of bits[i / 8] = (keep[i] != 0), least
  * significant bit first, the last byte padded with zeros.  bits: uint8 [(n + 7) / 8].
  */
 int pdd_pack_mask(const uint8_t* keep, int64_t n, uint8_t* bits, void* stream);
 
 /*
- * pdd_refine_vote -- per-head selection followed by a vote (Sec. 3.2 selects "the indices
- * with top values (with ratio r) per head" but sends one mask of the prompt's length; the
- * paper does not say how the per-head index sets are merged.  pdd_token_importance +
+ * pdd_refine_vote -- per-head selection followed by a vote (Sec. 3.2 takes, for every head,
+ * the indices with the largest values at ratio r, but sends one mask of the prompt's length;
+ * the paper does not say how the per-head index sets are merged.  pdd_token_importance +
  * pdd_refine_topk sum the heads first; this call is the other reading):
  *   1. every head h takes its own k candidates with the largest pooled column sums
  *      (candidates, k and tie rule exactly as in pdd_refine_topk);
@@ -276,8 +293,23 @@ int pdd_refine_from_colsum_static(const float* colsum, int64_t ld, int32_t n_hea
                                   double keep_ratio, uint8_t* keep, int32_t* n_kept,
                                   void* stream);
 
-/* Sticky device-side status of the handle (PDD_OK or PDD_ERR_TIMEOUT); synchronises `stream`. */
+/* Sticky device-side status of the handle (PDD_OK or PDD_ERR_TIMEOUT); synchronises `stream`.
+ * pdd_clear_status sets it back to PDD_OK (asynchronously on `stream`). */
 int pdd_status(pdd_kv* kv, void* stream, int32_t* sticky_device_status);
+int pdd_clear_status(pdd_kv* kv, void* stream);
+
+/*
+ * Self-tests of the error paths (not part of the hot path; the paper has no counterpart).
+ * pdd_selftest_wait_timeout enqueues a one-warp kernel that waits on a barrier nobody ever
+ *   arrives at, with a limit of limit_us microseconds (1..100000) instead of the hot kernels'
+ *   2 s; when the limit runs out the kernel raises the handle's sticky word exactly as a hot
+ *   kernel does (PDD_ERR_TIMEOUT) and returns normally.  Nothing hangs and nothing traps.
+ * pdd_debug_fail_launch makes the nth enqueue step (copy or kernel launch, counted from 1)
+ *   of the following hot calls on this handle report PDD_ERR_CUDA without being attempted;
+ *   0 disarms.  It exists to test that a failed call leaves the host state unchanged.
+ */
+int pdd_selftest_wait_timeout(pdd_kv* kv, uint32_t limit_us, void* stream);
+int pdd_debug_fail_launch(pdd_kv* kv, int32_t nth);
 
 /*
  * Diagnostics.  pdd_export_colsum copies a sequence's per-head column sums

@@ -24,7 +24,8 @@ EXPORTS = [
     "pdd_prefill_chunk", "pdd_append_received", "pdd_token_importance", "pdd_kv_kinds",
     "pdd_refine_topk", "pdd_refine_topk_batched", "pdd_refine_from_colsum_static", "pdd_refine_sentences", "pdd_pack_mask",
     "pdd_refine_vote", "pdd_refine_vote_workspace", "pdd_solve_rl",
-    "pdd_status", "pdd_export_colsum",
+    "pdd_status", "pdd_clear_status", "pdd_selftest_wait_timeout", "pdd_debug_fail_launch",
+    "pdd_export_colsum",
     "pdd_export_kv", "pdd_export_kinds", "pdd_last_lse", "pdd_trace_enable", "pdd_trace_read",
     "pdd_set_kernel_path", "pdd_set_schedule", "pdd_strerror", "pdd_last_error_detail",
 ]
@@ -97,6 +98,9 @@ def lib():
                                   vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.pdd_solve_rl.argtypes = [P(pdd_rl_problem), i32, P(pdd_rl_solution)]
     L.pdd_status.argtypes = [vp, vp, P(i32)]
+    L.pdd_clear_status.argtypes = [vp, vp]
+    L.pdd_selftest_wait_timeout.argtypes = [vp, u32, vp]
+    L.pdd_debug_fail_launch.argtypes = [vp, i32]
     L.pdd_export_colsum.argtypes = [vp, i32, vp, vp]
     L.pdd_export_kv.argtypes = [vp, i32, vp, vp, vp]
     L.pdd_export_kinds.argtypes = [vp, i32, vp, vp]
@@ -253,6 +257,18 @@ def pdd_status(h, stream) -> int:
     v = ctypes.c_int32(0)
     _check(lib().pdd_status(h, stream, ctypes.byref(v)), "pdd_status")
     return int(v.value)
+
+
+def pdd_clear_status(h, stream):
+    _check(lib().pdd_clear_status(h, stream), "pdd_clear_status")
+
+
+def pdd_selftest_wait_timeout(h, limit_us: int, stream):
+    _check(lib().pdd_selftest_wait_timeout(h, limit_us, stream), "pdd_selftest_wait_timeout")
+
+
+def pdd_debug_fail_launch(h, nth: int):
+    _check(lib().pdd_debug_fail_launch(h, nth), "pdd_debug_fail_launch")
 
 
 def pdd_export_colsum(h, seq_id, dst_ptr, stream):

@@ -15,19 +15,29 @@
 //
 // Roles inside a CTA:
 //   warp 0      TMA producer: Q tiles per pair, K and V blocks through two 2-stage rings
-//   warp 1      MMA issuer (one thread): S_t = Q_t K^T and O_t += P_t V with tcgen05.mma,
-//               interleaved over the two tiles so that one tile's softmax overlaps the
-//               other tile's MMAs (the warp also owns the TMEM allocation)
-//   warps 2-3   idle (they complete the control warpgroup)
+//   warp 1      MMA issuer of the scores (one thread): S_t(j) = Q_t K(j)^T with tcgen05.mma,
+//               S_0(j), S_1(j), S_0(j+1), ... (the warp also owns the TMEM allocation)
+//   warp 2      MMA issuer of the PV products (one thread): O_t += P_t(j) V(j).
+//               The scores of block j+1 do not wait for the PV product of block j (P has
+//               TMEM columns of its own), so a tile's softmax has a whole round of the other
+//               MMAs to finish in, and the tensor pipe, not the chain MMA -> softmax -> MMA,
+//               bounds the loop.  Two issuing threads, because each barrier wait costs the
+//               waiting thread ~100 cycles even when the barrier has completed, and the
+//               pipe's queue is too short to bridge that.
+//   warp 3      idle (it completes the control warpgroup)
 //   warps 4-7   softmax of tile 0 (one row per thread, the whole S row in registers),
 //               rescale of O_0, epilogue
 //   warps 8-11  the same for tile 1
 // The control warpgroup gives registers back (setmaxnreg.dec) and the two softmax
 // warpgroups take them (setmaxnreg.inc); the host checks the split against the kernel's
 // register count before the first launch, because a split above it would wait forever.
-// TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each (O uses head_dim);
-// P_t overwrites the first 64 columns of S_t as packed bf16 and is the TMEM A operand
-// of the PV product.  All waits are bounded; on expiry the kernel raises the sticky
+// TMEM (512 columns): S | P_0 | P_1 | O_0 | O_1.  S (128 fp32 columns) is shared by the two
+// tiles: a softmax warpgroup takes its whole row of S into registers as soon as it is
+// complete and hands the columns back (s_free), so they are free for the other tile's next
+// scores long before they are needed.  P_t (64 columns, packed bf16) has columns of its own
+// and is the TMEM A operand of the PV product; because it does not lie over S, the scores of
+// block j+1 can be computed while P_t(j) still waits for its PV product.  O_t: 128 columns
+// each (head_dim of them used).  All waits are bounded; on expiry the kernel raises the sticky
 // status word and every role leaves through the common exit that frees TMEM.
 #pragma once
 #include <type_traits>
@@ -70,6 +80,8 @@ struct AttnBars {
   uint64_t s_ready[2];    // MMA -> softmax: S_t(j) complete (and all earlier MMAs)
   uint64_t p_ready[2];    // softmax -> MMA: P_t(j) in TMEM, O_t rescaled
   uint64_t o_done[2];     // MMA -> softmax: last PV of tile t in this segment complete
+  uint64_t pv_done[2];    // MMA -> softmax: PV_t(j) complete (P_t may be overwritten, O_t rescaled)
+  uint64_t s_free;        // softmax -> MMA: the shared S columns have been read
   // cluster mode: x_full[t] collects, in every CTA, the other CTAs' "my export of tile t
   // stands"; x_free[t] their "I am done reading your export of tile t"
   uint64_t x_full[2], x_free[2];
@@ -246,6 +258,7 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
       ptx::mbar_init(&bars->s_ready[t], 1);
       ptx::mbar_init(&bars->p_ready[t], 128);
       ptx::mbar_init(&bars->o_done[t], 1);
+      ptx::mbar_init(&bars->pv_done[t], 1);
       ptx::mbar_init(&bars->x_full[t], kCluster && csize > 1 ? 128 * (csize - 1) : 1);
       ptx::mbar_init(&bars->x_free[t], kCluster && csize > 1 ? 128 * (csize - 1) : 1);
     }
@@ -255,6 +268,7 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
       ptx::mbar_init(&bars->v_full[s], 1);
       ptx::mbar_init(&bars->v_empty[s], 1);
     }
+    ptx::mbar_init(&bars->s_free, 128);
     bars->abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -355,66 +369,31 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
       }
       if (!ok) *abort_flag = 1;
     } else if (warp == 1 && lane == 0) {
-      // ---------------------------------------------------------------- MMA issuer
+      // ---------------------------------------------------------------- MMA issuer: scores
+      // S_t(j) = Q_t K(j)^T into the shared S columns, S_0(j), S_1(j), S_0(j+1), ...: each
+      // once the scores before it (the other tile's) have been taken into registers by their
+      // softmax warpgroup.  Nothing here depends on the PV products, which another thread
+      // issues: a barrier wait of one (~100 cycles even when it has completed) falls under the
+      // other's MMAs instead of leaving the tensor pipe idle.
       constexpr uint32_t idesc_qk = ptx::instr_desc_bf16(128, 128, 0, 0);
-      constexpr uint32_t idesc_pv = ptx::instr_desc_bf16(128, D, 0, 1);
-      const uint32_t q_addr = ptx::smem_u32(sQ), k_addr = ptx::smem_u32(sK),
-                     v_addr = ptx::smem_u32(sV);
       // Descriptors are built once; a K step only adds a constant to the address field.
-      const uint64_t dq0 = ptx::smem_desc_sw128(q_addr, 16, 1024);
-      const uint64_t dk0 = ptx::smem_desc_sw128(k_addr, 16, 1024);
-      const uint64_t dv0 = ptx::smem_desc_sw128(v_addr, L::kSubBytes, 1024);
-      auto issue_qk = [&](int t, int st) {
-        const uint32_t tS = tmem + 128 * t;
-        const uint64_t da = dq0 + (uint64_t)((t * L::kTileBytes) >> 4);
-        const uint64_t db = dk0 + (uint64_t)((st * L::kTileBytes) >> 4);
-        ptx::mma_ss_k64_first(tS, da, db, idesc_qk);
-        if (D == 128)      // second 64-column sub-tile of Q and K
-          ptx::mma_ss_k64_acc(tS, da + (L::kSubBytes >> 4), db + (L::kSubBytes >> 4), idesc_qk);
-      };
-      // half = 0: keys 0-63 of the block, half = 1: keys 64-127
-      auto issue_pv = [&](int t, int st, int half, bool first) {
-        ptx::mma_ts_k64(tmem + 256 + 128 * t, tmem + 128 * t + half * 32,
-                        dv0 + (uint64_t)((st * L::kTileBytes + half * 8192) >> 4), idesc_pv,
-                        first ? 0u : 1u);
-      };
-      // Everything this thread does between two MMAs delays the tensor pipe, so the loop
-      // state lives in scalars and the per-tile code is instantiated for t = 0 and t = 1.
+      const uint64_t dq0 = ptx::smem_desc_sw128(ptx::smem_u32(sQ), 16, 1024);
+      const uint64_t dk0 = ptx::smem_desc_sw128(ptx::smem_u32(sK), 16, 1024);
       SegmentWalk<kBand, kCluster> walk(rec, cta, csize, crank);
       Segment sg;
-      uint32_t kv_it = 0, q_cnt0 = 0, q_cnt1 = 0, blk0 = 0, blk1 = 0;
+      uint32_t kv_it = 0, q_cnt0 = 0, q_cnt1 = 0, n_qk = 0;
       bool ok = true;
-      bool k_next_ready = false, v_ready = false;
-      uint32_t st = 0, st1 = 1, ph = 0, ph1 = 0;
       const bool skip = wait_for_kernels_ahead();
-      // one key block of one tile: PV of its two halves, then the next S (or the end of the
-      // tile's share)
-      auto tile_step = [&](auto tc, int jj, int nb, uint32_t& blk) -> bool {
-        constexpr int t = decltype(tc)::value;
-        // All waits first, then PV (8 MMAs) and the next S (8 MMAs) as one uninterrupted
-        // run: the issuing thread pays a start-up for every group of MMAs it issues after a
-        // wait, and it is this thread, not the tensor pipe, that bounds the kernel.
-        const bool more = jj + 1 < nb;
-        if (!v_ready) {
-          if (!ptx::mbar_wait(&bars->v_full[st], ph)) return false;
-          v_ready = true;
-        }
-        if (more && !k_next_ready) {
-          if (!ptx::mbar_wait(&bars->k_full[st1], ph1)) return false;
-          k_next_ready = true;
-        }
-        if (!ptx::mbar_wait(&bars->p_ready[t], blk & 1)) return false;
-        ++blk;
+      auto qk = [&](int t, uint32_t st_k) -> bool {
+        if (n_qk > 0 && !ptx::mbar_wait(&bars->s_free, (n_qk - 1) & 1)) return false;
+        ++n_qk;
         ptx::tc_fence_after();
-        issue_pv(t, st, 0, jj == 0);
-        issue_pv(t, st, 1, false);
-        if (more) {
-          issue_qk(t, st1);
-          ptx::mma_commit(&bars->s_ready[t]);
-          if (jj + 2 == nb) ptx::mma_commit(&bars->q_empty[t]);
-        } else {
-          ptx::mma_commit(&bars->o_done[t]);
-        }
+        const uint64_t da = dq0 + (uint64_t)((t * L::kTileBytes) >> 4);
+        const uint64_t db = dk0 + (uint64_t)((st_k * L::kTileBytes) >> 4);
+        ptx::mma_ss_k64_first(tmem, da, db, idesc_qk);
+        if (D == 128)      // second 64-column sub-tile of Q and K
+          ptx::mma_ss_k64_acc(tmem, da + (L::kSubBytes >> 4), db + (L::kSubBytes >> 4), idesc_qk);
+        ptx::mma_commit(&bars->s_ready[t]);
         return true;
       };
       while (ok && !skip && walk.next(g, sg)) {
@@ -429,33 +408,55 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
           ok = ptx::mbar_wait(&bars->q_full[1], q_cnt1 & 1);
           ++q_cnt1;
         }
-        st = kv_it % kKvStages;
-        if (ok) ok = ptx::mbar_wait(&bars->k_full[st], (kv_it / kKvStages) & 1);
-        if (!ok) break;
+        for (int jj = 0; jj < nmax && ok; ++jj, ++kv_it) {
+          const uint32_t st = kv_it % kKvStages;
+          ok = ptx::mbar_wait(&bars->k_full[st], (kv_it / kKvStages) & 1);
+          if (ok && jj < nb0) {
+            ok = qk(0, st);
+            if (jj + 1 == nb0) ptx::mma_commit(&bars->q_empty[0]);
+          }
+          if (ok && jj < nb1) {
+            ok = qk(1, st);
+            if (jj + 1 == nb1) ptx::mma_commit(&bars->q_empty[1]);
+          }
+          ptx::mma_commit(&bars->k_empty[st]);
+        }
+      }
+      if (!ok) *abort_flag = 1;
+    } else if (warp == 2 && lane == 0) {
+      // ---------------------------------------------------------------- MMA issuer: PV products
+      // O_t (+)= P_t(j) V(j), tile 0 then tile 1 for every key block, each as soon as its
+      // softmax warpgroup has stored P_t(j).  tcgen05.commit covers the MMAs of the thread
+      // that executes it, so pv_done / o_done / v_empty follow the PV products alone.
+      constexpr uint32_t idesc_pv = ptx::instr_desc_bf16(128, D, 0, 1);
+      const uint64_t dv0 = ptx::smem_desc_sw128(ptx::smem_u32(sV), L::kSubBytes, 1024);
+      SegmentWalk<kBand, kCluster> walk(rec, cta, csize, crank);
+      Segment sg;
+      uint32_t kv_it = 0, blk0 = 0, blk1 = 0;
+      bool ok = true;
+      const bool skip = wait_for_kernels_ahead();
+      auto pv = [&](int t, uint32_t st_v, bool first, bool last, uint32_t& blk) -> bool {
+        if (!ptx::mbar_wait(&bars->p_ready[t], blk & 1)) return false;
+        ++blk;
         ptx::tc_fence_after();
-        if (nb0 > 0) {
-          issue_qk(0, st);
-          ptx::mma_commit(&bars->s_ready[0]);
-          if (nb0 == 1) ptx::mma_commit(&bars->q_empty[0]);
-        }
-        if (nb1 > 0) {
-          issue_qk(1, st);
-          ptx::mma_commit(&bars->s_ready[1]);
-          if (nb1 == 1) ptx::mma_commit(&bars->q_empty[1]);
-        }
-        ptx::mma_commit(&bars->k_empty[st]);
-        for (int jj = 0; jj < nmax; ++jj, ++kv_it) {
-          st = kv_it % kKvStages;
-          st1 = (kv_it + 1) % kKvStages;
-          ph = (kv_it / kKvStages) & 1;
-          ph1 = ((kv_it + 1) / kKvStages) & 1;
-          k_next_ready = false;
-          v_ready = false;
-          if (jj < nb0) ok = tile_step(std::integral_constant<int, 0>{}, jj, nb0, blk0);
-          if (ok && jj < nb1) ok = tile_step(std::integral_constant<int, 1>{}, jj, nb1, blk1);
-          if (!ok) break;
+        // keys 0-63 of the block, then keys 64-127
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+          ptx::mma_ts_k64(tmem + 256 + 128 * t, tmem + 128 + 64 * t + half * 32,
+                          dv0 + (uint64_t)((st_v * L::kTileBytes + half * 8192) >> 4), idesc_pv,
+                          (first && half == 0) ? 0u : 1u);
+        ptx::mma_commit(last ? &bars->o_done[t] : &bars->pv_done[t]);
+        return true;
+      };
+      while (ok && !skip && walk.next(g, sg)) {
+        const int nb0 = sg.nblk[0], nb1 = sg.nblk[1];
+        const int nmax = max(nb0, nb1);
+        for (int jj = 0; jj < nmax && ok; ++jj, ++kv_it) {
+          const uint32_t st = kv_it % kKvStages;
+          ok = ptx::mbar_wait(&bars->v_full[st], (kv_it / kKvStages) & 1);
+          if (ok && jj < nb0) ok = pv(0, st, jj == 0, jj + 1 == nb0, blk0);
+          if (ok && jj < nb1) ok = pv(1, st, jj == 0, jj + 1 == nb1, blk1);
           ptx::mma_commit(&bars->v_empty[st]);
-          if (k_next_ready) ptx::mma_commit(&bars->k_empty[st1]);
         }
       }
       if (!ok) *abort_flag = 1;
@@ -467,14 +468,15 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
     const int wq = warp & 3;                         // TMEM lane quarter of this warp
     const int r = wq * 32 + lane;                    // row of the tile
     const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
-    const uint32_t tS = tmem + 128 * t + lane_base;
+    const uint32_t tS = tmem + lane_base;                       // shared by the two tiles
+    const uint32_t tP = tmem + 128 + 64 * t + lane_base;
     const uint32_t tO = tmem + 256 + 128 * t + lane_base;
     const float sl2 = g.scale * 1.4426950408889634f;
     uint64_t* const bar_s = &bars->s_ready[t];
     uint64_t* const bar_p = &bars->p_ready[t];
     SegmentWalk<kBand, kCluster> walk(rec, cta, csize, crank);
     Segment sg;
-    int blk = 0, o_cnt = 0;
+    int blk = 0, o_cnt = 0, pv_cnt = 0;
     bool ok = !wait_for_kernels_ahead();     // (a skipped launch is not a failure: see below)
     const bool skipped = !ok;
     while (ok && walk.next(g, sg)) {
@@ -496,6 +498,9 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
 #pragma unroll
         for (int c4 = 0; c4 < 4; ++c4) ptx::tmem_ld32(tS + c4 * 32, s + c4 * 32);
         ptx::tmem_ld_wait();
+        // the S columns may take the next scores (the other tile's, as a rule)
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(&bars->s_free);
         if (need_mask) {     // only the block(s) on the diagonal: masked logits become -inf
           const int n_vis = min(kKeyBlock, p_row - key0 + 1);   // may be <= 0
 #pragma unroll
@@ -520,7 +525,21 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
         // A row that has seen no key yet has m = -inf; a share that starts on the diagonal
         // can leave it there for a whole block.
         const bool grow = bm > m && (m == -INFINITY || (bm - m) * sl2 > 8.f);
+        // PV_t(j-1) was issued after this block's scores: it must have completed before O_t is
+        // rescaled or P_t is overwritten.  The rescale (rare) waits here, the common path
+        // only before the store of P, when the product has long finished.
+        bool pv_waited = jj == 0;
+        auto wait_pv = [&]() -> bool {
+          if (pv_waited) return true;
+          pv_waited = true;
+          const bool got = ptx::mbar_wait(&bars->pv_done[t], (uint32_t)pv_cnt & 1);
+          ++pv_cnt;
+          ptx::tc_fence_after();
+          return got;
+        };
         if (__any_sync(0xffffffffu, grow)) {
+          ok = __all_sync(0xffffffffu, wait_pv());
+          if (!ok) break;
           const float m_new = fmaxf(m, bm);
           const float alpha = (m == -INFINITY) ? 0.f : ptx::ex2((m - m_new) * sl2);
           l *= alpha;
@@ -543,8 +562,8 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
         const float2 sl2v = make_float2(sl2, sl2);
         const float2 nmb = make_float2(-m_fin * sl2, -m_fin * sl2);
         float2 ps0 = make_float2(0.f, 0.f), ps1 = make_float2(0.f, 0.f);
-        // The first 64 keys are stored while the second 64 are exponentiated; one arrival
-        // hands the whole block to the MMA thread.  Off the diagonal half of the exponentials
+        // All of P is formed in registers first, then stored; one arrival hands the whole
+        // block to the MMA thread.  Off the diagonal half of the exponentials
         // are evaluated with a polynomial on the FMA pipe (kPolyExp), because the MUFU unit
         // (16 ex2 per clock per SM) is as loaded as the tensor pipe here: 128x128 ex2 per
         // tile and key block take as long as the tile's two MMAs.  Diagonal blocks keep the
@@ -569,13 +588,16 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
               s[c / 2] = *reinterpret_cast<uint32_t*>(&b0);
               s[c / 2 + 1] = *reinterpret_cast<uint32_t*>(&b1);
             }
-            ptx::tmem_st32(tS + 32 * half, s + 32 * half);
           }
         };
         if (need_mask || need_band || !kPolyExp)
           exp_block(std::false_type{});
         else
           exp_block(std::true_type{});
+        ok = __all_sync(0xffffffffu, wait_pv());
+        if (!ok) break;
+        ptx::tmem_st32(tP, s);
+        ptx::tmem_st32(tP + 32, s + 32);
         ptx::tmem_st_wait();
         ptx::tc_fence_before();
         ptx::mbar_arrive(bar_p);
@@ -783,6 +805,10 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
   ptx::tc_fence_before();
   __syncthreads();
   if (tid == 0 && *abort_flag) atomicExch(g.dev_status, 5);
+  // A CTA of a cluster must not leave while a peer may still read its shared memory (after a
+  // wait that ran out the x_free hand-shake of the merge can be cut short).  Every wait in
+  // this kernel is bounded, so every thread of every CTA of the cluster gets here.
+  if (kCluster) ptx::cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     ptx::tc_fence_after();

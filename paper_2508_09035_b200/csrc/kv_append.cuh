@@ -17,6 +17,8 @@ kv_append_kernel(CacheGeom g, void* __restrict__ rec_dev, const __grid_constant_
   // Only now may the attention kernel start: whatever it reads before its own wait (the
   // caller's q, cache rows of earlier calls) is then known to be complete.
   ptx::griddep_launch_dependents();
+  // a launch that follows a timed-out wait does no work (as in every kernel of the handle)
+  if (*reinterpret_cast<volatile int32_t*>(g.dev_status) != 0) return;
   const void* rec = rec_in_param ? reinterpret_cast<const void*>(&recp) : rec_dev;
   if (rec_in_param && blockIdx.x == 0) {
     const int n16 = (reinterpret_cast<const CallHeader*>(rec)->rec_bytes + 15) / 16;

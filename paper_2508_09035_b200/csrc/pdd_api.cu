@@ -130,9 +130,32 @@ struct pdd_kv {
   std::vector<int32_t> sched_nb;      // per-call scratch of the attention schedule
   std::vector<int64_t> sched_first;
   RecParam rec_param;                 // by-value copy of a small call record
+  int fail_countdown = 0;             // > 0: the n-th launch from now reports a failure (test hook)
 };
 
 namespace {
+
+// Test hook: true if this launch is the one that has been told to fail.
+bool injected_failure(pdd_kv* kv) {
+  if (kv->fail_countdown <= 0) return false;
+  return --kv->fail_countdown == 0;
+}
+
+// Waits on a barrier nobody arrives at; when the limit runs out it raises the sticky status
+// word like any hot kernel does and returns through the normal exit.
+__global__ void __launch_bounds__(32)
+wait_timeout_probe_kernel(int32_t* dev_status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_mbar_init();
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) {
+    const bool got = ptx::mbar_wait_for(&bar, 0, limit_ns, 0xf);
+    if (!got) atomicExch(dev_status, PDD_ERR_TIMEOUT);
+  }
+}
 
 struct Carve {
   size_t kpool, vpool, page_table, kinds, colsum, lse, status, part_o, part_ml, ring, total;
@@ -374,6 +397,27 @@ int run_call(pdd_kv* kv, const pdd_batch* b, const void* q, const void* k, const
   hdr.pages_off = (int32_t)(sizeof(CallHeader) + sizeof(SeqDesc) * (size_t)b->n_seqs);
   std::vector<SeqDesc> descs(b->n_seqs);
   int32_t* page_ids = reinterpret_cast<int32_t*>(rec_h + hdr.pages_off);
+  // The host state (lengths, page lists, free pages, ring position) moves forward while the
+  // record is built; if anything fails before the call's last launch has been accepted it is
+  // put back, so that a failed call leaves the handle as it found it.
+  struct Undo { int32_t seq; int64_t len; size_t n_pages; };
+  std::vector<Undo> undo;
+  undo.reserve(b->n_seqs);
+  const int ring_next_before = kv->ring_next;
+  const int64_t last_rows_before = kv->last_rows;
+  auto roll_back = [&](int rc) {
+    for (auto it = undo.rbegin(); it != undo.rend(); ++it) {
+      auto& pages = kv->seq_pages[it->seq];
+      while (pages.size() > it->n_pages) {
+        kv->free_pages.push_back(pages.back());
+        pages.pop_back();
+      }
+      kv->seq_len[it->seq] = it->len;
+    }
+    kv->ring_next = ring_next_before;
+    kv->last_rows = last_rows_before;
+    return rc;
+  };
   int tile0 = 0, page_off = 0, pair0 = 0;
   const int G = c.n_q_heads / c.n_kv_heads;
   for (int i = 0; i < b->n_seqs; ++i) {
@@ -392,6 +436,7 @@ int run_call(pdd_kv* kv, const pdd_batch* b, const void* q, const void* k, const
     if (d.len > 0) {
       const int64_t new_len = d.pos0 + d.len;
       const int64_t need = (new_len + c.page_tokens - 1) / c.page_tokens;
+      undo.push_back(Undo{s, kv->seq_len[s], kv->seq_pages[s].size()});
       while ((int64_t)kv->seq_pages[s].size() < need) {
         kv->seq_pages[s].push_back(kv->free_pages.back());
         kv->free_pages.pop_back();
@@ -542,8 +587,11 @@ int run_call(pdd_kv* kv, const pdd_batch* b, const void* q, const void* k, const
   if (rec_in_param) {
     memcpy(&recp, rec_h, used);
   } else {
-    PDD_CUDA(cudaMemcpyAsync(rec_d, rec_h, used, cudaMemcpyHostToDevice, st));
-    PDD_CUDA(cudaEventRecord(kv->ring_ev[slot], st));
+    cudaError_t ce = injected_failure(kv) ? cudaErrorUnknown
+                                          : cudaMemcpyAsync(rec_d, rec_h, used, cudaMemcpyHostToDevice, st);
+    if (ce == cudaSuccess) ce = cudaEventRecord(kv->ring_ev[slot], st);
+    if (ce != cudaSuccess)
+      return roll_back(fail(PDD_ERR_CUDA, "copy of the call record failed: %s", cudaGetErrorString(ce)));
     kv->ring_used[slot] = true;
   }
   // The device slots rotate in both cases: the slot's last readers are kernels of the call
@@ -557,17 +605,20 @@ int run_call(pdd_kv* kv, const pdd_batch* b, const void* q, const void* k, const
     Tracer t(kv, st, "kv_append");
     const int64_t n_vec = rows * c.n_kv_heads * c.head_dim / 8;
     const int blocks = (int)std::min<int64_t>((n_vec + 255) / 256, (int64_t)kv->sm_count * 8);
-    if (launch_pdl(kv_append_kernel, dim3(std::max(blocks, 1)), dim3(256), 0, st, kv->g,
+    if (injected_failure(kv) ||
+        launch_pdl(kv_append_kernel, dim3(std::max(blocks, 1)), dim3(256), 0, st, kv->g,
                    (void*)rec_d, recp, rec_in_param, (const __nv_bfloat16*)k,
                    (const __nv_bfloat16*)v) != cudaSuccess)
-      return fail(PDD_ERR_CUDA, "kv_append launch failed: %s",
-                  cudaGetErrorString(cudaGetLastError()));
+      return roll_back(fail(PDD_ERR_CUDA, "kv_append launch failed: %s",
+                            cudaGetErrorString(cudaGetLastError())));
   }
-  int rc = launch_attention(kv, rec_d, recp, rec_in_param, hdr, q, out, st);
-  if (rc) return rc;
+  int rc = injected_failure(kv) ? fail(PDD_ERR_CUDA, "fwd_attn launch failed: injected")
+                                : launch_attention(kv, rec_d, recp, rec_in_param, hdr, q, out, st);
+  if (rc) return roll_back(rc);
   if (flags & PDD_WINDOW) {
-    rc = launch_colsum(kv, rec_d, hdr, descs, q, st);
-    if (rc) return rc;
+    rc = injected_failure(kv) ? fail(PDD_ERR_CUDA, "colsum launch failed: injected")
+                              : launch_colsum(kv, rec_d, hdr, descs, q, st);
+    if (rc) return roll_back(rc);
   }
   return PDD_OK;
 }
@@ -636,7 +687,6 @@ int pdd_kv_alloc(const pdd_kv_config* cfg, void* dev_buf, size_t bytes, void* st
   pdd_kv* kv = new pdd_kv();
   kv->cfg = *cfg;
   if (kv->cfg.softmax_scale == 0.f) kv->cfg.softmax_scale = 1.f / sqrtf((float)cfg->head_dim);
-  // the arena may be handed in at any 256-byte boundary; the pools want 1024
   uint8_t* a = reinterpret_cast<uint8_t*>(dev_buf);
   kv->arena = a;
   kv->arena_bytes = bytes;
@@ -1020,6 +1070,29 @@ int pdd_status(pdd_kv* kv, void* stream, int32_t* sticky_device_status) {
   PDD_CUDA(cudaMemcpyAsync(&v, kv->g.dev_status, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
   PDD_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
   *sticky_device_status = v;
+  return PDD_OK;
+}
+
+int pdd_clear_status(pdd_kv* kv, void* stream) {
+  if (!kv) return fail(PDD_ERR_INVALID, "null handle");
+  PDD_CUDA(cudaMemsetAsync(kv->g.dev_status, 0, 4, (cudaStream_t)stream));
+  return PDD_OK;
+}
+
+int pdd_selftest_wait_timeout(pdd_kv* kv, uint32_t limit_us, void* stream) {
+  if (!kv) return fail(PDD_ERR_INVALID, "null handle");
+  if (limit_us == 0 || limit_us > 100000)
+    return fail(PDD_ERR_INVALID, "limit_us must be in 1..100000");
+  wait_timeout_probe_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(kv->g.dev_status,
+                                                              1000ull * limit_us);
+  PDD_CUDA(cudaGetLastError());
+  return PDD_OK;
+}
+
+int pdd_debug_fail_launch(pdd_kv* kv, int32_t nth) {
+  if (!kv) return fail(PDD_ERR_INVALID, "null handle");
+  if (nth < 0) return fail(PDD_ERR_INVALID, "nth must not be negative");
+  kv->fail_countdown = nth;
   return PDD_OK;
 }
 

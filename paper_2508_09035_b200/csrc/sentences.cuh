@@ -1,6 +1,9 @@
 // Sentence-level selection and the mask bit stream.
 //
-// refine_sentences_kernel: one CTA.  Sentence value = mean score of the sentence's prompt
+// refine_sentences_kernel: one CTA.  The sentence boundaries live in device memory, so the
+// host cannot check them: the kernel clamps every boundary to [0, n] and verifies that they
+// do not decrease; on a violation it keeps nothing, reports n_kept = -1 and returns (no index
+// derived from a bad boundary is ever used).  Sentence value = mean score of the sentence's prompt
 // tokens (added one by one in position order in fp32, then one division, so that the
 // decision can be repeated exactly on the host); sentences are sorted by decreasing value
 // (ties: lower sentence first) with a bitonic sort in shared memory, then taken first-fit
@@ -29,8 +32,26 @@ refine_sentences_kernel(const float* __restrict__ score, const uint8_t* __restri
   uint8_t* take = smem + (size_t)n_pad * 12;
   __shared__ int warp_buf[kSentenceThreads / 32];
   __shared__ int s_used;
+  __shared__ int s_bad;
   const int tid = threadIdx.x;
-  const int64_t lo = seg_start[0], hi = seg_start[n_seg];
+  // boundary s, clamped to [0, n]
+  auto bound = [&](int s) -> int64_t {
+    const int64_t b = seg_start[s];
+    return b < 0 ? 0 : (b > n ? n : b);
+  };
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+  for (int s = tid; s <= n_seg; s += kSentenceThreads) {
+    const int64_t b = seg_start[s];
+    if (b < 0 || b > n || (s > 0 && b < (int64_t)seg_start[s - 1])) s_bad = 1;
+  }
+  __syncthreads();
+  if (s_bad) {
+    for (int64_t i = tid; i < n; i += kSentenceThreads) keep[i] = 0;
+    if (tid == 0) *n_kept = -1;
+    return;
+  }
+  const int64_t lo = bound(0), hi = bound(n_seg);
 
   // prompt positions overall and inside the content range
   int c_prompt = 0, c_content = 0;
@@ -54,7 +75,7 @@ refine_sentences_kernel(const float* __restrict__ score, const uint8_t* __restri
     int c = 0;
     if (s < n_seg) {
       float acc = 0.f;
-      for (int i = seg_start[s]; i < seg_start[s + 1]; ++i) {
+      for (int64_t i = bound(s); i < bound(s + 1); ++i) {
         if (!kinds || kinds[i] == 0) {
           acc = __fadd_rn(acc, score[i]);
           ++c;
@@ -112,7 +133,7 @@ refine_sentences_kernel(const float* __restrict__ score, const uint8_t* __restri
   }
   for (int s = tid; s < n_seg; s += kSentenceThreads) {
     const uint8_t t = take[s];
-    for (int i = seg_start[s]; i < seg_start[s + 1]; ++i)
+    for (int64_t i = bound(s); i < bound(s + 1); ++i)
       keep[i] = (t && (!kinds || kinds[i] == 0)) ? 1 : 0;
   }
   if (tid == 0) *n_kept = n_always + s_used;
