@@ -3,12 +3,16 @@
 
 One "step" is one pass of the whole hot path over one synthetic prompt: every prefill
 chunk and the received-token append (KV append + causal attention + window column sums),
-then importance reduction and top-k keep mask.  The default workload is the
-Llama-7B-shaped layer: 32 query / 8 KV heads, head_dim 128, 4096-token prompt in chunks
-of 512 plus 64 received tokens, keep ratio 0.3.
+then importance reduction and top-k keep mask.  The default workload is the largest
+single-GPU configuration, the long prompt: 32 query / 8 KV heads, head_dim 128,
+32768-token prompt in chunks of 2048 plus 256 received tokens, 1 % outlier keys, keep
+ratio 0.2.  The same line carries an `also` list with the other configurations (the
+Llama-7B-shaped 4096-token layer, the 16 ragged sequences, and the 28-layer stack with its
+projection GEMMs done by torch and timed apart).  Short workloads repeat the pass inside a
+step so that the timed region spans enough clock samples whatever --steps is.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload c2|c4|c1|c5|c3l|c4s|c4w] [--window last|all]
+                  [--workload c4|c2|c5|c3|c1|c3l|c4s|c4w] [--window last|all] [--no-also]
 
 Prints ONE JSON line (rank 0).  `value` is tokens/s with inputs resident in HBM; `e2e`
 is the same metric through the C ABI with pinned-host inputs copied inside the timed
@@ -37,10 +41,14 @@ sys.path.insert(0, ROOT)
 from paper_2508_09035_b200 import workloads as wl  # noqa: E402
 
 NOMINAL_BF16_TFLOPS = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum of the attention kernel, mean over the launches of
-# one pass, from one ncu capture of this kernel on this workload (figures and command in
-# profiles/fwd_attn_c2_traffic.md).  Workloads without a capture report null.
-FWD_ATTN_DRAM_BYTES_PER_LAUNCH = {"c2": 14.15e6}
+# One ncu capture of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum of one
+# launch) on the small long-prompt case: the 2048-row chunk at pos0 = 6144 of an 8192-token
+# prompt.  DRAM traffic of this kernel grows in proportion to its algorithmic bytes (q + out +
+# one read of the sequence's K and V per call), so `roofline.traffic` scales the capture to the
+# mean launch of the timed workload.  The capture belongs to one version of the kernel source:
+# if csrc/attn_tc.cuh has changed since (first 12 hex digits of its sha256), traffic is null.
+FWD_ATTN_TRAFFIC_CAPTURE = dict(dram_bytes=None, algorithmic_bytes=None, source_sha256="")
+TARGET_TIMED_MS = 120.0          # a timed region at least this long (>= 20 clock samples at 4 ms)
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
 
@@ -64,6 +72,8 @@ def get_workload(name: str, window: str) -> wl.Workload:
         return wl.config_c4(window)
     if name == "c5":
         return wl.config_c5(window)
+    if name == "c3":
+        raise SystemExit("c3 is the layer stack: it has its own runner (StackRunner)")
     if name == "c3l":
         # One layer of config 3's attention stack (12 query / 2 KV heads, 8192-token prompt in
         # chunks of 1024, 128 received tokens after every chunk, every prompt row in the
@@ -458,17 +468,283 @@ def run_reference(args, rank: int, world: int):
     print(json.dumps(line), flush=True)
 
 
+def attention_source_tag() -> str:
+    import hashlib
+    path = os.path.join(ROOT, "paper_2508_09035_b200", "csrc", "attn_tc.cuh")
+    try:
+        return hashlib.sha256(open(path, "rb").read()).hexdigest()[:12]
+    except OSError:
+        return ""
+
+
+def attention_bytes_per_launch(w: wl.Workload) -> float:
+    """Algorithmic HBM bytes of the mean attention launch of a workload: q and out of the
+    call's rows plus one read of K and V of every sequence of the call up to its new length."""
+    per_row_q = w.n_q_heads * w.head_dim * 2
+    per_pos_kv = 2 * w.n_kv_heads * w.head_dim * 2
+    groups = grouped_calls(w)
+    total = 0
+    for _, _, group in groups:
+        for _, c in group:
+            total += 2 * c.length * per_row_q + (c.pos0 + c.length) * per_pos_kv
+    return total / max(len(groups), 1)
+
+
+def scaled_traffic(w: wl.Workload):
+    cap = FWD_ATTN_TRAFFIC_CAPTURE
+    if not cap["dram_bytes"] or cap["source_sha256"] != attention_source_tag():
+        return None
+    return cap["dram_bytes"] * attention_bytes_per_launch(w) / cap["algorithmic_bytes"]
+
+
+class StackRunner:
+    """Config 3: the 28-layer decoder attention stack.  Per call and layer:
+    x -> RMSNorm -> Wq, Wk, Wv (torch bf16 GEMMs) -> libpdd attention call -> Wo -> residual;
+    one pdd_kv handle per layer; importance accumulated over the layers, then one top-k.
+    The projections are glue, not part of the attention path: they are timed apart (the same
+    torch ops without the library calls) and counted in tokens/s only."""
+
+    def __init__(self, st: wl.LayerStack, device):
+        import ctypes
+        import torch
+        from paper_2508_09035_b200 import binding as B
+        self.torch, self.B, self.st, self.device = torch, B, st, device
+        self.lib = B.lib()
+        T = len(st.token_ids)
+        self.total_tokens = T
+        hq, hkv, d = st.n_q_heads, st.n_kv_heads, st.head_dim
+        self.max_rows = max(c.length for c in st.calls)
+        self.caches = [B.KVCache(hq, hkv, d, page_tokens=128, max_seqs=1, max_tokens_total=T,
+                                 max_tokens_per_seq=T, max_rows_per_call=self.max_rows,
+                                 device=device) for _ in range(st.n_layers)]
+        self.W = [{n: to_bf16_tensor(st.weight(l, n)).to(device) for n in "qkvo"}
+                  for l in range(st.n_layers)]
+        self.x_host = to_bf16_tensor(st.embedding_rows(st.token_ids), pin=True)
+        self.x_dev = self.x_host.to(device)
+        self.x_stage = torch.empty_like(self.x_dev)
+        self.out = torch.zeros((self.max_rows, hq, d), dtype=torch.bfloat16, device=device)
+        self.calls = []
+        for c in st.calls:
+            batch, keep = B.make_batch([0], [c.pos0], [c.length])
+            fn = self.lib.pdd_prefill_chunk if c.kind == wl.PROMPT else self.lib.pdd_append_received
+            self.calls.append(dict(fn=fn, batch=batch, keep=keep, bref=ctypes.byref(batch),
+                                   pos0=c.pos0, length=c.length,
+                                   flags=B.PDD_WINDOW if c.window else 0))
+        self.score = torch.zeros(T, dtype=torch.float32, device=device)
+        self.kinds = torch.from_numpy(st.kind.copy()).to(device)
+        self.keep = torch.empty(T, dtype=torch.uint8, device=device)
+        self.n_kept = torch.zeros(1, dtype=torch.int32, device=device)
+        self.keep_host = torch.empty(T, dtype=torch.uint8).pin_memory()
+        self.n_kept_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+        self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        self.h2d_bytes = self.x_host.numel() * 2
+        self.d2h_bytes = T + 4
+        self.stream = self.caches[0].stream
+        self.n_seqs = 1
+
+    def flush_l2(self):
+        self.flush_buf.fill_(1)
+
+    @staticmethod
+    def _rmsnorm(torch, x):
+        return torch.nn.functional.rms_norm(x, (x.shape[-1],), eps=1e-6)      # unit gain
+
+    def step(self, e2e: bool = False, attention: bool = True):
+        """One pass of the stack.  attention=False runs the glue alone (same torch ops, the
+        library calls left out) to time the projections."""
+        torch, B, lib, st = self.torch, self.B, self.lib, self.st
+        hq, hkv, d = st.n_q_heads, st.n_kv_heads, st.head_dim
+        rc = 0
+        if attention:
+            for cch in self.caches:
+                rc |= lib.pdd_kv_reset(cch.h, 0, self.stream)
+        if e2e:
+            self.x_stage.copy_(self.x_host, non_blocking=True)
+        x_all = self.x_stage if e2e else self.x_dev
+        for c in self.calls:
+            x = x_all[c["pos0"]:c["pos0"] + c["length"]]
+            out = self.out[:c["length"]]
+            for l, cch in enumerate(self.caches):
+                h_in = self._rmsnorm(torch, x)
+                W = self.W[l]
+                q = h_in @ W["q"]
+                k = h_in @ W["k"]
+                v = h_in @ W["v"]
+                if attention:
+                    rc |= c["fn"](cch.h, c["bref"], q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                  out.data_ptr(), c["flags"], self.stream)
+                x = torch.addmm(x, out.view(-1, hq * d), W["o"])
+        if attention:
+            for l, cch in enumerate(self.caches):
+                rc |= lib.pdd_token_importance(cch.h, 0, B.PDD_POOL_NONE, 1, self.score.data_ptr(),
+                                               1 if l > 0 else 0, self.stream)
+            rc |= lib.pdd_refine_topk(self.score.data_ptr(), self.kinds.data_ptr(),
+                                      self.total_tokens, 0, self.total_tokens,
+                                      float(st.keep_ratio), self.keep.data_ptr(),
+                                      self.n_kept.data_ptr(), self.stream)
+            if rc:
+                raise RuntimeError("libpdd call failed: %s" % lib.pdd_last_error_detail().decode())
+            if e2e:
+                self.keep_host.copy_(self.keep, non_blocking=True)
+                self.n_kept_host.copy_(self.n_kept, non_blocking=True)
+
+    def timed(self, steps: int, e2e: bool, passes: int = 1, attention: bool = True) -> float:
+        torch = self.torch
+        evs = []
+        for _ in range(steps * passes):
+            self.flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            self.step(e2e, attention)
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize(self.device)
+        return float(sum(a.elapsed_time(b) for a, b in evs))
+
+    def status(self) -> int:
+        return max(c.status() for c in self.caches)
+
+    def trace(self, on: bool):
+        for c in self.caches:
+            c.trace(on)
+
+    def trace_read(self) -> dict:
+        agg = {}
+        for c in self.caches:
+            for k, (n, ms) in c.trace_read().items():
+                a = agg.get(k, (0, 0.0))
+                agg[k] = (a[0] + n, a[1] + ms)
+        return agg
+
+    def attention_flops(self) -> int:
+        T = self.total_tokens
+        return 4 * self.st.head_dim * self.st.n_q_heads * (T * (T + 1) // 2) * self.st.n_layers
+
+
+def measure(name: str, window: str, steps: int, warmup: int, device, local: int, peaks,
+            world: int = 1, barrier=None) -> dict:
+    """Times one workload: HBM-resident passes, end-to-end passes, then a traced pass for the
+    per-kernel figures.  Returns the fields of a bench line (or of an `also` entry)."""
+    import torch
+    stack = name == "c3"
+    if stack:
+        st = wl.config_c3()
+        runner = StackRunner(st, device)
+        tokens, wname = runner.total_tokens, "c3_stack_%dl_l8192" % st.n_layers
+        description = ("%d-layer decoder attention stack, 12/2 heads, d=128, hidden 1536, 8192-token "
+                       "prompt in chunks of 1024 with 128 received tokens after each chunk, every "
+                       "prompt row in the observation window; RMSNorm + Wq/Wk/Wv/Wo by torch" % st.n_layers)
+        keep_ratio, flops, w = st.keep_ratio, runner.attention_flops(), None
+    else:
+        w = get_workload(name, window)
+        runner = Runner(w, device)
+        tokens, wname, description = w.n_tokens, w.name, w.description
+        keep_ratio, flops = w.keep_ratio, w.attention_flops()
+    barrier = barrier or (lambda: torch.cuda.synchronize(device))
+
+    for _ in range(warmup):
+        runner.step(False)
+        runner.step(True)
+    torch.cuda.synchronize(device)
+    # how many passes make one step: short workloads repeat the pass so that the timed region
+    # is long enough for the clock record
+    t0 = time.perf_counter()
+    runner.step(False)
+    torch.cuda.synchronize(device)
+    est_ms = max((time.perf_counter() - t0) * 1e3, 1e-3)
+    passes = max(1, int(np.ceil(TARGET_TIMED_MS / (est_ms * steps))))
+    sampler = ClockSampler(local, str(getattr(torch.cuda.get_device_properties(device), "uuid", "")))
+    sampler.start()
+    barrier()
+    sampler.mark()
+    ms_dev = runner.timed(steps, False, passes) if stack else runner.timed(steps * passes, e2e=False)
+    barrier()
+    ms_e2e = runner.timed(steps, True, passes) if stack else runner.timed(steps * passes, e2e=True)
+    barrier()
+    sampler.mark()
+    clocks = sampler.stop()
+    status = runner.status() if stack else runner.kv.status()
+    assert status == 0, "device-side error word set"
+    n_kept = int(runner.n_kept_host.sum().item())
+    glue_ms = None
+    if stack:
+        glue_ms = runner.timed(min(steps, 2), False, 1, attention=False) / min(steps, 2)
+
+    # per-kernel timing pass (events around every launch; not part of the numbers above)
+    trace_steps = min(steps * passes, 2 if stack else 5)
+    if stack:
+        runner.trace(True)
+        for _ in range(trace_steps):
+            runner.flush_l2()
+            torch.cuda._sleep(int(1.9e6))
+            runner.step(False)
+            torch.cuda.synchronize(device)
+        trace = runner.trace_read()
+        runner.trace(False)
+    else:
+        runner.kv.trace(True)
+        runner.topk_events = []
+        for _ in range(trace_steps):
+            runner.flush_l2()
+            runner.backlog(1.0)
+            runner.step(False)
+            torch.cuda.synchronize(device)
+        trace = runner.kv.trace_read()
+        runner.kv.trace(False)
+        trace["radix_topk"] = (len(runner.topk_events),
+                               float(sum(a.elapsed_time(b) for a, b in runner.topk_events)))
+        runner.topk_events = None
+    launches_per_pass = sum(c for c, _ in trace.values()) // trace_steps
+    attn_name = "fwd_attn" if "fwd_attn" in trace else sorted(
+        (k for k in trace if k.startswith("attn")), key=lambda k: -trace[k][1])[0]
+    attn_cnt, attn_ms = trace[attn_name]
+    flops_per_launch = flops / (attn_cnt / trace_steps)
+    attn_tflops = flops_per_launch / (attn_ms / attn_cnt * 1e-3) / 1e12
+    comb_ms = trace.get("attn_combine", (0, 0.0))[1]
+    attn_with_combine = flops * trace_steps / ((attn_ms + comb_ms) * 1e-3) / 1e12
+
+    n_passes = steps * passes
+    ms_dev_all, units = aggregate_over_ranks(ms_dev, tokens * n_passes, world, device)
+    ms_e2e_all, _ = aggregate_over_ranks(ms_e2e, tokens * n_passes, world, device)
+    res = dict(
+        workload=wname, description=description, tokens_per_pass=tokens, passes_per_step=passes,
+        value=units / (ms_dev_all * 1e-3), ms_per_step=ms_dev_all / steps,
+        ms_per_pass=ms_dev_all / n_passes,
+        e2e=dict(value=units / (ms_e2e_all * 1e-3), unit="tokens/s",
+                 h2d_bytes_per_step=runner.h2d_bytes * passes,
+                 d2h_bytes_per_step=runner.d2h_bytes * passes, ms_per_step=ms_e2e_all / steps),
+        attention_tflops=attn_tflops, attention_tflops_with_combine=attn_with_combine,
+        frac_of_measured_peak=attn_tflops / peaks["bf16"],
+        frac_of_nominal_peak=attn_tflops / NOMINAL_BF16_TFLOPS,
+        launches_per_pass=int(launches_per_pass), clocks=clocks, n_kept=n_kept,
+        keep_ratio=keep_ratio, attn_kernel=attn_name,
+        kernels=(kernel_table(trace, trace_steps, w, peaks) if w is not None else
+                 {k: dict(launches=c, total_ms=ms) for k, (c, ms) in trace.items()}),
+        traffic=scaled_traffic(w) if w is not None else None,
+        _workload=w)
+    if stack:
+        res["projection_glue_ms_per_pass"] = glue_ms
+        res["attention_path_ms_per_pass"] = max(ms_dev_all / n_passes - glue_ms, 0.0)
+    del runner
+    torch.cuda.empty_cache()
+    return res
+
+
+ALSO_WORKLOADS = (("c2", 20), ("c5", 4), ("c3", 2))     # name, steps (each step repeats short passes)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--workload", default="c4")
     ap.add_argument("--window", default="last", choices=["last", "all"])
     ap.add_argument("--ref-stride", type=int, default=0)
     ap.add_argument("--cpu-baseline-stride", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-also", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -485,9 +761,6 @@ def main():
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
     peaks = load_peaks()
-    w = get_workload(args.workload, args.window)
-    runner = Runner(w, device)
-    tokens = w.n_tokens
 
     def barrier():
         if world > 1:
@@ -495,79 +768,61 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(device)
 
-    for _ in range(args.warmup):
-        runner.step(False)
-        runner.step(True)
-    sampler = ClockSampler(local, str(getattr(torch.cuda.get_device_properties(device), "uuid", "")))
-    sampler.start()
-    barrier()
-    sampler.mark()
-    ms_dev = runner.timed(args.steps, e2e=False)
-    barrier()
-    ms_e2e = runner.timed(args.steps, e2e=True)
-    barrier()
-    sampler.mark()
-    clocks = sampler.stop()
-    assert runner.kv.status() == 0, "device-side error word set"
-    n_kept = int(runner.n_kept_host.sum().item())
-
-    # per-kernel timing pass (events around every launch; not part of the numbers above)
-    runner.kv.trace(True)
-    runner.topk_events = []
-    trace_steps = min(args.steps, 5)
-    for _ in range(trace_steps):
-        runner.flush_l2()
-        runner.backlog(1.0)
-        runner.step(False)
-        torch.cuda.synchronize(device)
-    trace = runner.kv.trace_read()
-    runner.kv.trace(False)
-    trace["radix_topk"] = (len(runner.topk_events),
-                           float(sum(a.elapsed_time(b) for a, b in runner.topk_events)))
-    runner.topk_events = None
-    launches_per_step = sum(c for c, _ in trace.values()) // trace_steps
-    attn_name = "fwd_attn" if "fwd_attn" in trace else sorted(
-        (k for k in trace if k.startswith("attn")), key=lambda k: -trace[k][1])[0]
-    attn_cnt, attn_ms = trace[attn_name]
-    flops_per_launch = w.attention_flops() / (attn_cnt / trace_steps)
-    achieved_tflops = flops_per_launch / (attn_ms / attn_cnt * 1e-3) / 1e12
-    # the same with the merge of shared key ranges counted in
-    comb_ms = trace.get("attn_combine", (0, 0.0))[1]
-    attn_with_combine_tflops = w.attention_flops() * trace_steps / ((attn_ms + comb_ms) * 1e-3) / 1e12
-
-    ms_dev_all, units = aggregate_over_ranks(ms_dev, tokens * args.steps, world, device)
-    ms_e2e_all, _ = aggregate_over_ranks(ms_e2e, tokens * args.steps, world, device)
+    m = measure(args.workload, args.window, args.steps, args.warmup, device, local, peaks, world,
+                barrier)
+    also = []
+    if not args.no_also and world == 1:
+        for name, k in ALSO_WORKLOADS:
+            if name == args.workload:
+                continue
+            a = measure(name, args.window, k, 3, device, local, peaks)
+            also.append(dict(
+                workload=a["workload"], value=a["value"], unit="tokens/s",
+                ms_per_step=a["ms_per_step"], ms_per_pass=a["ms_per_pass"],
+                passes_per_step=a["passes_per_step"], steps=k,
+                e2e_value=a["e2e"]["value"], attention_tflops=a["attention_tflops"],
+                attention_tflops_with_combine=a["attention_tflops_with_combine"],
+                frac=a["frac_of_measured_peak"], frac_of_nominal_peak=a["frac_of_nominal_peak"],
+                launches_per_pass=a["launches_per_pass"], clocks=a["clocks"],
+                **({"projection_glue_ms_per_pass": a["projection_glue_ms_per_pass"],
+                    "attention_path_ms_per_pass": a["attention_path_ms_per_pass"]}
+                   if "projection_glue_ms_per_pass" in a else {})))
     if rank != 0:
         return
-    value = units / (ms_dev_all * 1e-3)
-    e2e_value = units / (ms_e2e_all * 1e-3)
+    w = m["_workload"]
     line = dict(
-        metric="prefill_tokens_per_s", value=value, unit="tokens/s", n_gpus=world,
-        steps=args.steps, warmup=args.warmup, ms_per_step=ms_dev_all / args.steps,
+        metric="prefill_tokens_per_s", value=m["value"], unit="tokens/s", n_gpus=world,
+        steps=args.steps, warmup=args.warmup, ms_per_step=m["ms_per_step"],
         higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
-        config=dict(workload=w.name, description=w.description, window=args.window,
-                    keep_ratio=w.keep_ratio, l2="flushed between steps (256 MiB write)",
+        config=dict(workload=m["workload"], description=m["description"], window=args.window,
+                    keep_ratio=m["keep_ratio"], passes_per_step=m["passes_per_step"],
+                    l2="flushed between passes (256 MiB write)",
                     e2e_copies="pinned host -> device per call on a copy stream, overlapped with "
-                               "the previous call's kernels; keep mask read back",
-                    parallelism="replicas only" if world > 1 else "1 gpu", n_kept=n_kept),
-        attention_tflops=achieved_tflops,
-        attention_tflops_with_combine=attn_with_combine_tflops,
-        attention_frac_of_nominal_peak=achieved_tflops / NOMINAL_BF16_TFLOPS,
-        e2e=dict(value=e2e_value, unit="tokens/s", h2d_bytes_per_step=runner.h2d_bytes,
-                 d2h_bytes_per_step=runner.d2h_bytes, ms_per_step=ms_e2e_all / args.steps),
-        gpu_launches=int(launches_per_step * args.steps),
-        clocks=clocks,
-        kernels=kernel_table(trace, trace_steps, w, peaks),
-        roofline=dict(bound="tensor", kernel=attn_name, achieved=achieved_tflops,
-                      peak=peaks["bf16"], unit="TFLOP/s", frac=achieved_tflops / peaks["bf16"],
+                               "the previous call's kernels; keep mask read back; the attention "
+                               "output stays on the device (the next layer reads it there)",
+                    parallelism="replicas only" if world > 1 else "1 gpu", n_kept=m["n_kept"]),
+        attention_tflops=m["attention_tflops"],
+        attention_tflops_with_combine=m["attention_tflops_with_combine"],
+        attention_frac_of_nominal_peak=m["frac_of_nominal_peak"],
+        e2e=m["e2e"],
+        gpu_launches=int(m["launches_per_pass"] * m["passes_per_step"] * args.steps),
+        clocks=m["clocks"],
+        kernels=m["kernels"],
+        roofline=dict(bound="tensor", kernel=m["attn_kernel"], achieved=m["attention_tflops"],
+                      peak=peaks["bf16"], unit="TFLOP/s", frac=m["frac_of_measured_peak"],
                       peak_source=peaks["source"] + " burst bf16 (kernel timed alone per launch)",
-                      frac_of_sustained_peak=(achieved_tflops / peaks["bf16_sustained"]
+                      frac_of_sustained_peak=(m["attention_tflops"] / peaks["bf16_sustained"]
                                               if peaks["bf16_sustained"] else None),
-                      traffic=FWD_ATTN_DRAM_BYTES_PER_LAUNCH.get(args.workload),
-                      traffic_unit="bytes per launch (dram read + write, mean over the pass)"),
+                      traffic=m["traffic"],
+                      traffic_unit="bytes per launch (dram read + write of one ncu capture of this "
+                                   "kernel, scaled by algorithmic bytes to the mean launch)"),
+        also=also,
     )
-    if not args.no_cpu_baseline:
-        # whole prompt for the short workloads (a few seconds), every n-th row for the long ones
+    if m.get("projection_glue_ms_per_pass") is not None:
+        line["projection_glue_ms_per_pass"] = m["projection_glue_ms_per_pass"]
+    if not args.no_cpu_baseline and w is not None:
+        # a bounded sample: whole prompt for the short workloads, every n-th row for the long ones
+        tokens = w.n_tokens
         stride = args.cpu_baseline_stride or (1 if tokens <= 8192 else tokens // 2048)
         n, dt, cores = oracle_sample(w, stride)
         line["cpu_baseline"] = dict(value=n / dt, unit="tokens/s", cores=cores, kind="oracle",
