@@ -21,6 +21,9 @@
 namespace pdd {
 
 constexpr int kColsumThreads = 192;
+// Pairs of every 4 whose exp2 is a polynomial on the FMA pipe (measured on the long-prompt
+// window pass: 0 -> 0.83 ms, 1 -> 0.78, 2 -> 0.80, 3 -> 0.91).
+constexpr int kColsumPoly = 1;
 
 __device__ __forceinline__ float ex2f_cs(float x) {
   float y;
@@ -51,7 +54,7 @@ struct ColsumBars {
 
 template <int D>
 __global__ void __launch_bounds__(kColsumThreads, 2)
-colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int seq_slot, int hsplit,
+colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
                  const __grid_constant__ CUtensorMap tmQ,
                  const __grid_constant__ CUtensorMap tmK) {
   using L = ColsumSmem<D>;
@@ -69,11 +72,23 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int seq_slot, int hs
   // (their LSE rows and cache rows are needed anyway).
   ptx::griddep_launch_dependents();
   ptx::griddep_wait();
-  const SeqDesc sd = record_descs(rec)[seq_slot];
+  // blockIdx.x runs over the key blocks of all window sequences of the call, one after another
+  const CallHeader* hdr = reinterpret_cast<const CallHeader*>(rec);
+  const SeqDesc* descs = record_descs(rec);
+  int kt = blockIdx.x, seq_slot = 0;
+  for (; seq_slot < hdr->n_seqs; ++seq_slot) {
+    const SeqDesc& d = descs[seq_slot];
+    if (!d.window || d.len <= 0) continue;
+    const int n_kb = (int)((d.pos0 + d.len + kKeyBlock - 1) / kKeyBlock);
+    if (kt < n_kb) break;
+    kt -= n_kb;
+  }
+  if (seq_slot >= hdr->n_seqs) return;
+  const SeqDesc sd = descs[seq_slot];
   const int G = g.hq / g.hkv;
   // blockIdx.y = (KV head, part): with few key blocks and KV heads the query heads of a group
   // are dealt out to `hsplit` CTAs (each still the only writer of its heads' column sums)
-  const int kt = blockIdx.x, kvh = blockIdx.y / hsplit;
+  const int kvh = blockIdx.y / hsplit;
   const int hpc = G / hsplit;                                   // query heads per CTA
   const int h_first = kvh * G + (blockIdx.y % hsplit) * hpc;
   const int64_t key0 = (int64_t)kt * kKeyBlock;
@@ -131,15 +146,19 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int seq_slot, int hs
                            kvh, page);
       }
       bool ok = true;
+      int h = h_first, qt = qt_min;
       for (int it = 0; it < n_items && ok; ++it) {
         const int st = it & 1;
-        const int h = h_first + it / n_qt_act, qt = qt_min + it % n_qt_act;
         if (it >= 2) ok = ptx::mbar_wait(&bars->q_empty[st], (uint32_t)((it >> 1) - 1) & 1);
         if (!ok) break;
         ptx::mbar_expect_tx(&bars->q_full[st], L::kTileBytes);
         for (int sub = 0; sub < L::kSub; ++sub)
           ptx::tma_load_3d(sQ + st * L::kTileBytes + sub * L::kSubBytes, &tmQ, &bars->q_full[st],
                            64 * sub, h, (int)(sd.tok_offset + (int64_t)qt * kTileRows));
+        if (++qt == qt_end) {
+          qt = qt_min;
+          ++h;
+        }
       }
       if (!ok) *abort_flag = 1;
     }
@@ -177,23 +196,38 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int seq_slot, int hs
     float acc = 0.f;
     int cur_h = h_first;
     bool ok = true;
-    for (int it = 0; it < n_items; ++it) {
+    // LSE (exp2 domain) of the rows of an item's query tile; fetched one item ahead so that the
+    // global-memory latency falls under the previous item's exponentials.
+    auto fetch_lse = [&](int h, int qt) -> float {
+      const int rows_valid = min(kTileRows, sd.len - qt * kTileRows);
+      const int64_t row0 = sd.tok_offset + (int64_t)qt * kTileRows;
+      return ct < rows_valid ? g.lse[(size_t)h * g.lse_ld + row0 + ct] * 1.4426950408889634f : 0.f;
+    };
+    // item it = (head h_first + it / n_qt_act, query tile qt_min + it % n_qt_act), stepped
+    // without divisions; (hn, qn) is the item after it
+    int h = h_first, qt = qt_min, hn = h_first, qn = qt_min;
+    float lse_next = fetch_lse(h, qt);
+    for (int it = 0; it < n_items; ++it, h = hn, qt = qn) {
       const int st = it & 1;
       const uint32_t ph = (uint32_t)(it >> 1) & 1;
-      const int h = h_first + it / n_qt_act, qt = qt_min + it % n_qt_act;
+      qn = qt + 1;
+      hn = h;
+      if (qn == qt_end) {
+        qn = qt_min;
+        ++hn;
+      }
       if (h != cur_h) {
         if (key < T) g.colsum[((size_t)sd.seq_id * g.hq + cur_h) * g.max_tokens_per_seq + key] += acc;
         acc = 0.f;
         cur_h = h;
       }
       const int rows_valid = min(kTileRows, sd.len - qt * kTileRows);
-      const int64_t row0 = sd.tok_offset + (int64_t)qt * kTileRows;
       const int64_t pq0 = sd.pos0 + (int64_t)qt * kTileRows;     // position of query column 0
-      // LSE of the tile's rows, in the exp2 domain, broadcast through shared memory
-      sLse[st * 128 + ct] = ct < rows_valid
-                                ? g.lse[(size_t)h * g.lse_ld + row0 + ct] * 1.4426950408889634f
-                                : 0.f;
+      // (the stage's previous reader, item it-2, finished before this thread arrived on
+      // s_empty for it, and every thread's arrival precedes the MMA that precedes s_full)
+      sLse[st * 128 + ct] = lse_next;
       ptx::mbar_arrive(&bars->lse_ready[st]);
+      if (it + 1 < n_items) lse_next = fetch_lse(hn, qn);
       ok = ptx::mbar_wait(&bars->lse_ready[st], ph);
       if (ok) ok = ptx::mbar_wait(&bars->s_full[st], ph);
       ok = __all_sync(0xffffffffu, ok);
@@ -201,27 +235,69 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int seq_slot, int hs
       ptx::tc_fence_after();
       const bool full = rows_valid == kTileRows && pq0 >= key0 + kKeyBlock - 1 &&
                         pq0 + kTileRows - 1 - key0 < g.window;
-      const float* ls = sLse + st * 128;
+      // LSE of the 32 columns in hand, as eight 16-byte shared-memory loads (every thread of
+      // the warp reads the same words: one broadcast each).  Going through the generic float
+      // pointer instead costs one load instruction per exponential, and those loads, not the
+      // MUFU unit, then bound the kernel.
+      const uint32_t ls_addr = ptx::smem_u32(sLse + st * 128);
+      // 32 query columns at a time; the next 32 are on their way while these are
+      // exponentiated, and the accumulator goes back to the MMA thread as soon as the last
+      // ones have landed in registers.  Two partial sums, added in a fixed order.
+      float acc0 = 0.f, acc1 = 0.f;
+      auto add32 = [&](int c4, const uint32_t* v) {
+        float ls[32];
 #pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) {
-        uint32_t v[32];
-        ptx::tmem_ld32(tmem + 128 * st + lane_base + c4 * 32, v);
-        ptx::tmem_ld_wait();
+        for (int i = 0; i < 8; ++i)
+          asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                       : "=f"(ls[4 * i]), "=f"(ls[4 * i + 1]), "=f"(ls[4 * i + 2]), "=f"(ls[4 * i + 3])
+                       : "r"(ls_addr + (uint32_t)(c4 * 128 + i * 16)));
         if (full) {
+          // The MUFU unit (16 exponentials per clock per SM) bounds this loop, so kColsumPoly
+          // of every 4 pairs go through a cubic on the FMA pipe instead (7.5e-5 relative
+          // error against a 1e-2 bound on the sums).
 #pragma unroll
-          for (int c = 0; c < 32; ++c)
-            acc += ex2f_cs(fmaf(__uint_as_float(v[c]), sl2, -ls[c4 * 32 + c]));
+          for (int c = 0; c < 32; c += 8) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float x0 = fmaf(__uint_as_float(v[c + 2 * i]), sl2, -ls[c + 2 * i]);
+              const float x1 = fmaf(__uint_as_float(v[c + 2 * i + 1]), sl2, -ls[c + 2 * i + 1]);
+              if (i < kColsumPoly) {
+                const float2 e = ptx::ex2_poly2(make_float2(x0, x1));
+                acc0 += e.x;
+                acc1 += e.y;
+              } else {
+                acc0 += ex2f_cs(x0);
+                acc1 += ex2f_cs(x1);
+              }
+            }
+          }
         } else {
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
             const int col = c4 * 32 + c;
-            const float e = ex2f_cs(fmaf(__uint_as_float(v[c]), sl2, -ls[col]));
-            acc += (col < rows_valid && pq0 + col >= key && pq0 + col - key < g.window) ? e : 0.f;
+            const float e = ex2f_cs(fmaf(__uint_as_float(v[c]), sl2, -ls[c]));
+            const float ee = (col < rows_valid && pq0 + col >= key && pq0 + col - key < g.window) ? e : 0.f;
+            if (c & 1) acc1 += ee; else acc0 += ee;
           }
         }
-      }
+      };
+      const uint32_t tacc = tmem + 128 * st + lane_base;
+      uint32_t va[32], vb[32];
+      ptx::tmem_ld32(tacc, va);
+      ptx::tmem_ld_wait();
+      ptx::tmem_ld32(tacc + 32, vb);
+      add32(0, va);
+      ptx::tmem_ld_wait();
+      ptx::tmem_ld32(tacc + 64, va);
+      add32(1, vb);
+      ptx::tmem_ld_wait();
+      ptx::tmem_ld32(tacc + 96, vb);
+      add32(2, va);
+      ptx::tmem_ld_wait();
       ptx::tc_fence_before();
       ptx::mbar_arrive(&bars->s_empty[st]);
+      add32(3, vb);
+      acc += acc0 + acc1;
     }
     if (ok && key < T)
       g.colsum[((size_t)sd.seq_id * g.hq + cur_h) * g.max_tokens_per_seq + key] += acc;
@@ -248,26 +324,24 @@ inline cudaError_t prepare_colsum_tc(int d) {
                                          ColsumSmem<64>::kBytes);
 }
 
-inline cudaError_t launch_colsum_tc(const CacheGeom& g, const void* rec_dev, int seq_slot,
-                                    const SeqDesc& sd, const CUtensorMap& tmQ,
-                                    const CUtensorMap& tmK, int sm_count, cudaStream_t st) {
-  const int64_t T = sd.pos0 + sd.len;
-  const int n_kb = (int)((T + kKeyBlock - 1) / kKeyBlock);
+// One launch for all window sequences of a call: n_kb_total = their key blocks, added up.
+inline cudaError_t launch_colsum_tc(const CacheGeom& g, const void* rec_dev, int n_kb_total,
+                                    const CUtensorMap& tmQ, const CUtensorMap& tmK, int sm_count,
+                                    cudaStream_t st) {
+  if (n_kb_total <= 0) return cudaSuccess;
   // Two CTAs fit on an SM.  When (key blocks x KV heads) leaves most of those slots empty, the
   // heads of a GQA group go to separate CTAs: the largest divisor of the group size that
   // still fits one wave (the K tile is then fetched once per part, from L2).
   const int G = g.hq / g.hkv, slots = 2 * sm_count;
   int hsplit = 1;
   for (int s = 2; s <= G; ++s)
-    if (G % s == 0 && (int64_t)n_kb * g.hkv * s <= slots) hsplit = s;
-  dim3 grid((unsigned)n_kb, (unsigned)(g.hkv * hsplit));
+    if (G % s == 0 && (int64_t)n_kb_total * g.hkv * s <= slots) hsplit = s;
+  dim3 grid((unsigned)n_kb_total, (unsigned)(g.hkv * hsplit));
   if (g.d == 128)
     return launch_pdl(colsum_tc_kernel<128>, grid, dim3(kColsumThreads), ColsumSmem<128>::kBytes,
-                      st, g, rec_dev, seq_slot, hsplit, tmQ, tmK);
-  else
-    return launch_pdl(colsum_tc_kernel<64>, grid, dim3(kColsumThreads), ColsumSmem<64>::kBytes,
-                      st, g, rec_dev, seq_slot, hsplit, tmQ, tmK);
-  return cudaGetLastError();
+                      st, g, rec_dev, hsplit, tmQ, tmK);
+  return launch_pdl(colsum_tc_kernel<64>, grid, dim3(kColsumThreads), ColsumSmem<64>::kBytes,
+                    st, g, rec_dev, hsplit, tmQ, tmK);
 }
 
 }  // namespace pdd

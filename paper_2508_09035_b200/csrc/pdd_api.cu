@@ -325,12 +325,12 @@ int launch_colsum(pdd_kv* kv, const void* rec_dev, const CallHeader& hdr,
   if (rc) return rc;
   const CUtensorMap& tmQ = *tmq_ptr;
   Tracer t(kv, st, "colsum");
-  for (int s = 0; s < hdr.n_seqs; ++s) {
-    if (!descs[s].window || descs[s].len == 0) continue;
-    if (launch_colsum_tc(g, rec_dev, s, descs[s], tmQ, kv->tmK, kv->sm_count, st) != cudaSuccess)
-      return fail(PDD_ERR_CUDA, "colsum launch failed: %s",
-                  cudaGetErrorString(cudaGetLastError()));
-  }
+  int n_kb_total = 0;
+  for (int s = 0; s < hdr.n_seqs; ++s)
+    if (descs[s].window && descs[s].len > 0)
+      n_kb_total += (int)((descs[s].pos0 + descs[s].len + kKeyBlock - 1) / kKeyBlock);
+  if (launch_colsum_tc(g, rec_dev, n_kb_total, tmQ, kv->tmK, kv->sm_count, st) != cudaSuccess)
+    return fail(PDD_ERR_CUDA, "colsum launch failed: %s", cudaGetErrorString(cudaGetLastError()));
   return PDD_OK;
 }
 
