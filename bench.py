@@ -306,6 +306,7 @@ class Runner:
         self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)
         self.d2h_bytes = n + 4 * self.n_seqs
         self.stream = self.kv.stream
+        self.seq_ids = (ctypes.c_int32 * self.n_seqs)(*range(self.n_seqs))
         self.topk_args = ((ctypes.c_int64 * (self.n_seqs + 1))(*self.offsets),
                           (ctypes.c_int64 * self.n_seqs)(*([0] * self.n_seqs)),
                           (ctypes.c_int64 * self.n_seqs)(*[s.n_tokens for s in w.seqs]))
@@ -350,19 +351,24 @@ class Runner:
             else:
                 q, k, v = c["dev_ptrs"]
             rc |= c["fn"](h, c["bref"], q, k, v, c["out_ptr"], c["flags"], st)
-        for si in range(self.n_seqs):
-            rc |= lib.pdd_token_importance(h, si, B.PDD_POOL_NONE, 1,
-                                           self.score.data_ptr() + 4 * self.offsets[si], 0, st)
-        if self.topk_events is not None:      # the handle-free top-k is not in the library's trace
-            ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-            ev[0].record()
-        rc |= lib.pdd_refine_topk_batched(self.score.data_ptr(), self.kinds.data_ptr(), self.n_seqs,
-                                          self.topk_args[0], self.topk_args[1], self.topk_args[2],
-                                          float(w.keep_ratio), self.keep.data_ptr(),
-                                          self.n_kept.data_ptr(), st)
-        if self.topk_events is not None:
-            ev[1].record()
-            self.topk_events.append(ev)
+        if self.n_seqs == 1:
+            # one sequence: importance reduction and selection through one call
+            rc |= lib.pdd_importance_topk(h, 0, B.PDD_POOL_NONE, 1, self.score.data_ptr(), 0, 0,
+                                          self.total_tokens, float(w.keep_ratio),
+                                          self.keep.data_ptr(), self.n_kept.data_ptr(), st)
+        else:
+            rc |= lib.pdd_token_importance_batched(h, self.n_seqs, self.seq_ids, B.PDD_POOL_NONE, 1,
+                                                   self.score.data_ptr(), self.topk_args[0], 0, st)
+            if self.topk_events is not None:  # the handle-free top-k is not in the library's trace
+                ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                ev[0].record()
+            rc |= lib.pdd_refine_topk_batched(self.score.data_ptr(), self.kinds.data_ptr(),
+                                              self.n_seqs, self.topk_args[0], self.topk_args[1],
+                                              self.topk_args[2], float(w.keep_ratio),
+                                              self.keep.data_ptr(), self.n_kept.data_ptr(), st)
+            if self.topk_events is not None:
+                ev[1].record()
+                self.topk_events.append(ev)
         if rc:
             raise RuntimeError("libpdd call failed: %s" % lib.pdd_last_error_detail().decode())
         if e2e:
@@ -397,9 +403,9 @@ def kernel_table(trace, trace_steps: int, w: wl.Workload, peaks) -> dict:
         "kv_append": 2 * n_tokens * row_kv + n_tokens,
         # read fp32 column sums of every head, write one fp32 score per position
         "importance_reduce": 4 * n_tokens * (w.n_q_heads + 1),
-        # counting pass, four radix passes and the mask pass read score (fp32) and kind (1 byte)
-        # of every position; the mask pass writes one byte
-        "radix_topk": n_tokens * (6 * 5 + 1),
+        # scores (fp32) read once into shared memory; kind (1 byte) read by the counting pass,
+        # the four radix passes and the mask pass; the mask pass writes one byte
+        "radix_topk": n_tokens * (4 + 6 + 1),
     }
     out = {}
     for k, (c, ms) in trace.items():
@@ -691,8 +697,9 @@ def measure(name: str, window: str, steps: int, warmup: int, device, local: int,
             torch.cuda.synchronize(device)
         trace = runner.kv.trace_read()
         runner.kv.trace(False)
-        trace["radix_topk"] = (len(runner.topk_events),
-                               float(sum(a.elapsed_time(b) for a, b in runner.topk_events)))
+        if runner.topk_events:
+            trace["radix_topk"] = (len(runner.topk_events),
+                                   float(sum(a.elapsed_time(b) for a, b in runner.topk_events)))
         runner.topk_events = None
     launches_per_pass = sum(c for c, _ in trace.values()) // trace_steps
     attn_name = "fwd_attn" if "fwd_attn" in trace else sorted(

@@ -142,6 +142,25 @@ int pdd_append_received(pdd_kv* kv, const pdd_batch* batch, const void* q, const
 int pdd_token_importance(pdd_kv* kv, int32_t seq_id, int32_t pool_kind, int32_t pool_k,
                          float* score, int32_t accumulate, void* stream);
 
+/*
+ * pdd_token_importance_batched -- the same for several sequences in one launch: sequence
+ * seq_ids[i] writes (or adds to) score[offsets[i] .. offsets[i+1]-1]; offsets[i+1]-offsets[i]
+ * must equal its length.  seq_ids, offsets: HOST arrays.
+ *
+ * pdd_importance_topk -- pdd_token_importance followed by pdd_refine_topk for one sequence in
+ * one call (Sec. 3.2: sum, pooling, top values), with the position kinds taken from the
+ * cache: two kernels chained on the stream, the second starting under the first's tail.
+ * Results are bit-identical to the two calls.  (Selections of at most 49152 positions per
+ * sequence, through any of the top-k calls, stage the scores in shared memory and read them
+ * from global memory once; longer ones read them once per radix pass.)
+ */
+int pdd_token_importance_batched(pdd_kv* kv, int32_t n_seqs, const int32_t* seq_ids,
+                                 int32_t pool_kind, int32_t pool_k, float* score,
+                                 const int64_t* offsets, int32_t accumulate, void* stream);
+int pdd_importance_topk(pdd_kv* kv, int32_t seq_id, int32_t pool_kind, int32_t pool_k,
+                        float* score, int32_t accumulate, int64_t cand_lo, int64_t cand_hi,
+                        double keep_ratio, uint8_t* keep, int32_t* n_kept, void* stream);
+
 /* Device pointer to a sequence's kind array (uint8 [length]); valid until pdd_kv_free. */
 int pdd_kv_kinds(pdd_kv* kv, int32_t seq_id, const uint8_t** kinds);
 

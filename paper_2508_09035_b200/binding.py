@@ -21,7 +21,8 @@ PATH_TENSOR_CORE, PATH_SIMT, PATH_TENSOR_CORE_SIMPLE = 0, 1, 2
 
 EXPORTS = [
     "pdd_kv_bytes_required", "pdd_kv_alloc", "pdd_kv_free", "pdd_kv_reset", "pdd_kv_length",
-    "pdd_prefill_chunk", "pdd_append_received", "pdd_token_importance", "pdd_kv_kinds",
+    "pdd_prefill_chunk", "pdd_append_received", "pdd_token_importance",
+    "pdd_token_importance_batched", "pdd_importance_topk", "pdd_kv_kinds",
     "pdd_refine_topk", "pdd_refine_topk_batched", "pdd_refine_from_colsum_static", "pdd_refine_sentences", "pdd_pack_mask",
     "pdd_refine_vote", "pdd_refine_vote_workspace", "pdd_solve_rl",
     "pdd_status", "pdd_clear_status", "pdd_selftest_wait_timeout", "pdd_debug_fail_launch",
@@ -85,6 +86,9 @@ def lib():
     for f in (L.pdd_prefill_chunk, L.pdd_append_received):
         f.argtypes = [vp, P(pdd_batch), vp, vp, vp, vp, u32, vp]
     L.pdd_token_importance.argtypes = [vp, i32, i32, i32, vp, i32, vp]
+    L.pdd_token_importance_batched.argtypes = [vp, i32, P(i32), i32, i32, vp, P(i64), i32, vp]
+    L.pdd_importance_topk.argtypes = [vp, i32, i32, i32, vp, i32, i64, i64, ctypes.c_double,
+                                      vp, vp, vp]
     L.pdd_kv_kinds.argtypes = [vp, i32, P(vp)]
     L.pdd_refine_topk.argtypes = [vp, vp, i64, i64, i64, ctypes.c_double, vp, vp, vp]
     L.pdd_refine_topk_batched.argtypes = [vp, vp, i32, P(i64), P(i64), P(i64), ctypes.c_double,
@@ -179,6 +183,22 @@ def pdd_append_received(h, batch, q_ptr, k_ptr, v_ptr, out_ptr, flags, stream):
 def pdd_token_importance(h, seq_id, pool_kind, pool_k, score_ptr, accumulate, stream):
     _check(lib().pdd_token_importance(h, seq_id, pool_kind, pool_k, score_ptr, accumulate, stream),
            "pdd_token_importance")
+
+
+def pdd_token_importance_batched(h, seq_ids, pool_kind, pool_k, score_ptr, offsets, accumulate,
+                                 stream):
+    n = len(seq_ids)
+    a_id = (ctypes.c_int32 * n)(*seq_ids)
+    a_off = (ctypes.c_int64 * (n + 1))(*offsets)
+    _check(lib().pdd_token_importance_batched(h, n, a_id, pool_kind, pool_k, score_ptr, a_off,
+                                              accumulate, stream), "pdd_token_importance_batched")
+
+
+def pdd_importance_topk(h, seq_id, pool_kind, pool_k, score_ptr, accumulate, cand_lo, cand_hi,
+                        keep_ratio, keep_ptr, n_kept_ptr, stream):
+    _check(lib().pdd_importance_topk(h, seq_id, pool_kind, pool_k, score_ptr, accumulate, cand_lo,
+                                     cand_hi, keep_ratio, keep_ptr, n_kept_ptr, stream),
+           "pdd_importance_topk")
 
 
 def pdd_kv_kinds(h, seq_id) -> int:

@@ -45,24 +45,50 @@ kv_append_kernel(CacheGeom g, void* __restrict__ rec_dev, const __grid_constant_
 
   const uint4* k4 = reinterpret_cast<const uint4*>(k);
   const uint4* v4 = reinterpret_cast<const uint4*>(v);
-  const int vec_per_head = g.d / 8;
-  for (int64_t i = tid; i < n_vec; i += stride) {
-    int64_t row = i / vec_per_row;
-    int rem = (int)(i - row * vec_per_row);
-    int kvh = rem / vec_per_head;
-    int c = rem - kvh * vec_per_head;
-    // sequence of this packed row (few sequences per call: linear scan)
-    int s = 0;
-    while (s + 1 < n_seqs && descs[s + 1].tok_offset <= row) ++s;
-    const SeqDesc& sd = descs[s];
-    int64_t pos = sd.pos0 + (row - sd.tok_offset);
-    int e = (int)(pos / g.page_tokens) - (int)(sd.pos0 / g.page_tokens);
-    int32_t page = pages[sd.page_off + e];
-    size_t dst = ((((size_t)page * g.hkv + kvh) * g.page_tokens + (size_t)(pos % g.page_tokens)) *
-                  g.d) / 8 + c;
-    reinterpret_cast<uint4*>(g.kpool)[dst] = k4[i];
-    reinterpret_cast<uint4*>(g.vpool)[dst] = v4[i];
-    if (rem == 0) g.kinds[(size_t)sd.seq_id * g.max_tokens_per_seq + pos] = (uint8_t)hdr->kind;
+  const uint32_t vec_per_head = (uint32_t)g.d / 8;
+  const uint32_t vpr = (uint32_t)vec_per_row;
+  const uint32_t page_tokens = (uint32_t)g.page_tokens;
+  // destination of vector i (32-bit index arithmetic: a call carries far fewer than 2^31
+  // vectors); the sequence of a packed row is found by a scan that starts at the sequence of
+  // the thread's previous vector (rows only grow along a thread's stride)
+  int s_hint = 0;
+  auto dest = [&](uint32_t i, bool& first_of_row, size_t& kind_at) -> size_t {
+    const uint32_t row = i / vpr, rem = i - row * vpr;
+    const uint32_t kvh = rem / vec_per_head, c = rem - kvh * vec_per_head;
+    while (s_hint + 1 < n_seqs && descs[s_hint + 1].tok_offset <= (int64_t)row) ++s_hint;
+    const SeqDesc& sd = descs[s_hint];
+    const uint32_t pos = (uint32_t)sd.pos0 + (row - (uint32_t)sd.tok_offset);
+    const uint32_t e = pos / page_tokens - (uint32_t)sd.pos0 / page_tokens;
+    const int32_t page = pages[sd.page_off + e];
+    first_of_row = rem == 0;
+    kind_at = (size_t)sd.seq_id * g.max_tokens_per_seq + pos;
+    return ((((size_t)page * g.hkv + kvh) * page_tokens + pos % page_tokens) * g.d) / 8 + c;
+  };
+  // four vectors of K and of V in flight per thread before the first store
+  constexpr int kUnroll = 4;
+  const uint32_t n = (uint32_t)n_vec, t0 = (uint32_t)tid, step = (uint32_t)stride;
+  for (uint32_t base = t0; base < n; base += kUnroll * step) {
+    uint4 kk[kUnroll], vv[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const uint32_t i = base + u * step;
+      if (i < n) {
+        kk[u] = k4[i];
+        vv[u] = v4[i];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const uint32_t i = base + u * step;
+      if (i < n) {
+        bool first;
+        size_t kind_at;
+        const size_t dst = dest(i, first, kind_at);
+        reinterpret_cast<uint4*>(g.kpool)[dst] = kk[u];
+        reinterpret_cast<uint4*>(g.vpool)[dst] = vv[u];
+        if (first) g.kinds[kind_at] = (uint8_t)hdr->kind;
+      }
+    }
   }
 }
 

@@ -178,6 +178,8 @@ int validate_cfg(const pdd_kv_config* c) {
     return fail(PDD_ERR_INVALID, "token capacities must be positive");
   if (c->max_tokens_per_seq > (1 << 24))
     return fail(PDD_ERR_UNSUPPORTED, "max_tokens_per_seq above 2^24");
+  if (c->max_rows_per_call > (1 << 22))
+    return fail(PDD_ERR_UNSUPPORTED, "max_rows_per_call above 2^22");
   if (c->sliding_window < 0 || c->reserved_f != 0.f || c->softmax_scale < 0.f)
     return fail(PDD_ERR_INVALID, "sliding_window >= 0, reserved_f must be 0, softmax_scale >= 0");
   return PDD_OK;
@@ -604,7 +606,7 @@ int run_call(pdd_kv* kv, const pdd_batch* b, const void* q, const void* k, const
   {
     Tracer t(kv, st, "kv_append");
     const int64_t n_vec = rows * c.n_kv_heads * c.head_dim / 8;
-    const int blocks = (int)std::min<int64_t>((n_vec + 255) / 256, (int64_t)kv->sm_count * 8);
+    const int blocks = (int)std::min<int64_t>((n_vec / 4 + 255) / 256, (int64_t)kv->sm_count * 8);
     if (injected_failure(kv) ||
         launch_pdl(kv_append_kernel, dim3(std::max(blocks, 1)), dim3(256), 0, st, kv->g,
                    (void*)rec_d, recp, rec_in_param, (const __nv_bfloat16*)k,
@@ -832,6 +834,65 @@ int pdd_token_importance(pdd_kv* kv, int32_t seq_id, int32_t pool_kind, int32_t 
   return PDD_OK;
 }
 
+int pdd_token_importance_batched(pdd_kv* kv, int32_t n_seqs, const int32_t* seq_ids,
+                                 int32_t pool_kind, int32_t pool_k, float* score,
+                                 const int64_t* offsets, int32_t accumulate, void* stream) {
+  if (!kv || !score || !seq_ids || !offsets) return fail(PDD_ERR_INVALID, "null argument");
+  if (n_seqs <= 0) return fail(PDD_ERR_INVALID, "n_seqs must be positive");
+  if (pool_kind < 0 || pool_kind > 2) return fail(PDD_ERR_INVALID, "pool_kind must be 0, 1 or 2");
+  if (pool_k < 1 || pool_k % 2 == 0 || pool_k > 1025)
+    return fail(PDD_ERR_INVALID, "pool_k must be odd and in 1..1025");
+  for (int i = 0; i < n_seqs; ++i) {
+    if (seq_ids[i] < 0 || seq_ids[i] >= kv->cfg.max_seqs)
+      return fail(PDD_ERR_INVALID, "seq_id out of range");
+    if (offsets[i + 1] - offsets[i] != kv->seq_len[seq_ids[i]])
+      return fail(PDD_ERR_INVALID, "offsets[%d+1] - offsets[%d] differs from the sequence's length", i, i);
+  }
+  const CacheGeom& g = kv->g;
+  cudaStream_t st = (cudaStream_t)stream;
+  Tracer t(kv, st, "importance_reduce");
+  for (int base = 0; base < n_seqs; base += kImportanceBatch) {
+    ImportanceBatch ib{};
+    const int cnt = std::min(kImportanceBatch, n_seqs - base);
+    int64_t n_max = 0;
+    for (int i = 0; i < cnt; ++i) {
+      const int32_t s = seq_ids[base + i];
+      ib.colsum[i] = g.colsum + (size_t)s * g.hq * g.max_tokens_per_seq;
+      ib.score[i] = score + offsets[base + i];
+      ib.n[i] = kv->seq_len[s];
+      n_max = std::max(n_max, ib.n[i]);
+    }
+    if (n_max == 0) continue;
+    PDD_CUDA(launch_pdl(importance_reduce_batched_kernel, dim3((unsigned)((n_max + 255) / 256), cnt),
+                        dim3(256), 0, st, ib, (int64_t)g.max_tokens_per_seq, (int)g.hq,
+                        pool_k == 1 ? 0 : pool_kind, pool_k, accumulate));
+  }
+  return PDD_OK;
+}
+
+int pdd_importance_topk(pdd_kv* kv, int32_t seq_id, int32_t pool_kind, int32_t pool_k,
+                        float* score, int32_t accumulate, int64_t cand_lo, int64_t cand_hi,
+                        double keep_ratio, uint8_t* keep, int32_t* n_kept, void* stream) {
+  if (!kv || !keep || !n_kept) return fail(PDD_ERR_INVALID, "null argument");
+  if (seq_id < 0 || seq_id >= kv->cfg.max_seqs) return fail(PDD_ERR_INVALID, "seq_id out of range");
+  if (pool_kind < 0 || pool_kind > 2) return fail(PDD_ERR_INVALID, "pool_kind must be 0, 1 or 2");
+  if (pool_k < 1 || pool_k % 2 == 0 || pool_k > 1025)
+    return fail(PDD_ERR_INVALID, "pool_k must be odd and in 1..1025");
+  if (!(keep_ratio >= 0.0 && keep_ratio <= 1.0))
+    return fail(PDD_ERR_INVALID, "keep_ratio must be in [0,1]");
+  const int64_t n = kv->seq_len[seq_id];
+  if (n <= 0) return fail(PDD_ERR_STATE, "the sequence is empty");
+  if (cand_lo < 0 || cand_hi > n || cand_lo > cand_hi)
+    return fail(PDD_ERR_INVALID, "candidate range outside [0,n]");
+  if (!score) return fail(PDD_ERR_INVALID, "score must not be null");
+  const CacheGeom& g = kv->g;
+  const uint8_t* kinds = g.kinds + (size_t)seq_id * g.max_tokens_per_seq;
+  int rc = pdd_token_importance(kv, seq_id, pool_kind, pool_k, score, accumulate, stream);
+  if (rc) return rc;
+  Tracer t(kv, (cudaStream_t)stream, "radix_topk");
+  return pdd_refine_topk(score, kinds, n, cand_lo, cand_hi, keep_ratio, keep, n_kept, stream);
+}
+
 int pdd_kv_kinds(pdd_kv* kv, int32_t seq_id, const uint8_t** kinds) {
   if (!kv || !kinds) return fail(PDD_ERR_INVALID, "null argument");
   if (seq_id < 0 || seq_id >= kv->cfg.max_seqs) return fail(PDD_ERR_INVALID, "seq_id out of range");
@@ -855,6 +916,20 @@ int pdd_refine_topk_batched(const float* score, const uint8_t* kinds, int32_t n_
       return fail(PDD_ERR_INVALID, "sequence %d: candidate range outside [0,n]", i);
   }
   cudaStream_t st = (cudaStream_t)stream;
+  int64_t n_max = 0;
+  for (int i = 0; i < n_seqs; ++i) n_max = std::max(n_max, offsets[i + 1] - offsets[i]);
+  const bool staged = n_max <= kStagedTopkMax;
+  if (staged) {
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    PDD_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < kMaxDevices && !attr_set[dev]) {
+      PDD_CUDA(cudaFuncSetAttribute(radix_topk_staged_kernel,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)(kStagedTopkMax * 4)));
+      attr_set[dev] = true;
+    }
+  }
   for (int base = 0; base < n_seqs; base += kTopkBatch) {
     TopkBatch tb{};
     const int cnt = std::min(kTopkBatch, n_seqs - base);
@@ -865,8 +940,13 @@ int pdd_refine_topk_batched(const float* score, const uint8_t* kinds, int32_t n_
       tb.s[i].cand_lo = cand_lo[base + i];
       tb.s[i].cand_hi = cand_hi[base + i];
     }
-    PDD_CUDA(launch_pdl(radix_topk_kernel<ScoreKeys>, dim3(cnt), dim3(kTopkThreads), 0, st,
-                        ScoreKeys{score}, kinds, tb, keep_ratio, keep, n_kept + base));
+    if (staged)
+      PDD_CUDA(launch_pdl(radix_topk_staged_kernel, dim3(cnt), dim3(kTopkThreads),
+                          (size_t)std::max<int64_t>(n_max, 1) * 4, st, score, kinds, tb, keep_ratio,
+                          keep, n_kept + base));
+    else
+      PDD_CUDA(launch_pdl(radix_topk_kernel<ScoreKeys>, dim3(cnt), dim3(kTopkThreads), 0, st,
+                          ScoreKeys{score}, kinds, tb, keep_ratio, keep, n_kept + base));
   }
   return PDD_OK;
 }

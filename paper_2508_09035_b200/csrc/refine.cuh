@@ -8,6 +8,52 @@
 
 namespace pdd {
 
+// score of position j: per-head pooled column sums added over the heads in index order
+__device__ __forceinline__ float pooled_head_sum(const float* __restrict__ colsum, int64_t ld,
+                                                 int hq, int64_t n, int pool_kind, int pool_k,
+                                                 int64_t j) {
+  const int half = pool_k / 2;
+  const int64_t lo = max((int64_t)0, j - half), hi = min(n - 1, j + half);
+  float total = 0.f;
+  for (int h = 0; h < hq; ++h) {
+    const float* cs = colsum + (size_t)h * ld;
+    float r;
+    if (pool_kind == 2) {
+      r = -INFINITY;
+      for (int64_t t = lo; t <= hi; ++t) r = fmaxf(r, cs[t]);
+    } else if (pool_kind == 1) {
+      r = 0.f;
+      for (int64_t t = lo; t <= hi; ++t) r += cs[t];
+      r /= (float)pool_k;                       // zero padding, fixed divisor
+    } else {
+      r = cs[j];
+    }
+    total += r;
+  }
+  return total;
+}
+
+// Several sequences in one launch: blockIdx.y = sequence of the batch.
+constexpr int kImportanceBatch = 64;
+struct ImportanceBatch {
+  const float* colsum[kImportanceBatch];   // [hq][ld] of the sequence
+  float* score[kImportanceBatch];
+  int64_t n[kImportanceBatch];
+};
+__global__ void __launch_bounds__(256)
+importance_reduce_batched_kernel(const ImportanceBatch b, int64_t ld, int hq, int pool_kind,
+                                 int pool_k, int accumulate) {
+  ptx::griddep_launch_dependents();
+  ptx::griddep_wait();
+  const int s = blockIdx.y;
+  const int64_t n = b.n[s];
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= n) return;
+  const float total = pooled_head_sum(b.colsum[s], ld, hq, n, pool_kind, pool_k, j);
+  float* score = b.score[s];
+  score[j] = accumulate ? score[j] + total : total;
+}
+
 __global__ void __launch_bounds__(256)
 importance_reduce_kernel(const float* __restrict__ colsum, int64_t ld, int hq, int64_t n,
                          int pool_kind, int pool_k, float* __restrict__ score, int accumulate) {
@@ -83,19 +129,18 @@ __device__ __forceinline__ int block_sum(int v, int* warp_buf) {
   return t;
 }
 
+// Selection of one sequence by the whole CTA (kTopkThreads threads): the body of
+// radix_topk_kernel, also used by the fused importance + selection kernel.
 template <class Keys>
-__global__ void __launch_bounds__(kTopkThreads)
-radix_topk_kernel(const Keys keys, const uint8_t* __restrict__ kinds,
-                  const TopkBatch seqs, double keep_ratio,
-                  uint8_t* __restrict__ keep, int32_t* __restrict__ n_kept) {
+__device__ __forceinline__ void radix_topk_body(const Keys& keys, const uint8_t* __restrict__ kinds,
+                                                const TopkSeq& sq, double keep_ratio,
+                                                uint8_t* __restrict__ keep,
+                                                int32_t* __restrict__ n_kept_out) {
   using key_t = typename Keys::key_t;
   __shared__ int hist[256];
   __shared__ int warp_buf[kTopkThreads / 32];
   __shared__ key_t s_prefix;
   __shared__ int s_need;
-  ptx::griddep_launch_dependents();
-  ptx::griddep_wait();          // see importance_reduce_kernel
-  const TopkSeq sq = seqs.s[blockIdx.x];
   const uint8_t* kd = kinds ? kinds + sq.kinds_offset : nullptr;
   uint8_t* kp = keep + sq.offset;
   const int tid = threadIdx.x;
@@ -203,7 +248,45 @@ radix_topk_kernel(const Keys keys, const uint8_t* __restrict__ kinds,
     }
     __syncthreads();
   }
-  if (tid == 0) n_kept[blockIdx.x] = k + n_always;
+  if (tid == 0) *n_kept_out = k + n_always;
+}
+
+template <class Keys>
+__global__ void __launch_bounds__(kTopkThreads)
+radix_topk_kernel(const Keys keys, const uint8_t* __restrict__ kinds,
+                  const TopkBatch seqs, double keep_ratio,
+                  uint8_t* __restrict__ keep, int32_t* __restrict__ n_kept) {
+  ptx::griddep_launch_dependents();
+  ptx::griddep_wait();          // see importance_reduce_kernel
+  radix_topk_body(keys, kinds, seqs.s[blockIdx.x], keep_ratio, keep, n_kept + blockIdx.x);
+}
+
+// Keys held in shared memory (filled by the fused kernel below): read from global memory once.
+struct SmemScoreKeys {
+  using key_t = uint32_t;
+  static constexpr int kPasses = 4;
+  const uint32_t* key;
+  __device__ __forceinline__ key_t load(int64_t i) const { return key[i]; }
+};
+
+// Selection with the keys staged in shared memory: a CTA reads its sequence's scores from
+// global memory once (n * 4 bytes of dynamic shared memory, at most kStagedTopkMax positions per
+// sequence) and the four radix passes and the mask pass work on the staged keys.
+constexpr int64_t kStagedTopkMax = 49152;       // positions (192 KiB of keys)
+__global__ void __launch_bounds__(kTopkThreads)
+radix_topk_staged_kernel(const float* __restrict__ score, const uint8_t* __restrict__ kinds,
+                         const TopkBatch seqs, double keep_ratio, uint8_t* __restrict__ keep,
+                         int32_t* __restrict__ n_kept) {
+  extern __shared__ __align__(16) uint32_t s_key[];
+  ptx::griddep_launch_dependents();
+  ptx::griddep_wait();
+  TopkSeq sq = seqs.s[blockIdx.x];
+  const float* sc = score + sq.offset;
+  for (int64_t j = threadIdx.x; j < sq.n; j += kTopkThreads) s_key[j] = order_key(sc[j]);
+  __syncthreads();
+  uint8_t* kp = keep + sq.offset;
+  sq.offset = 0;                 // keys and mask are addressed from the sequence's start
+  radix_topk_body(SmemScoreKeys{s_key}, kinds, sq, keep_ratio, kp, n_kept + blockIdx.x);
 }
 
 }  // namespace pdd

@@ -311,3 +311,66 @@ def test_empty_sequences_inside_a_batch():
         H.check_importance(cs, want_cs, H.imp_atol(T, hq, T) / hq, "seq %d colsum" % si)
     assert kv.status() == 0
     kv.close()
+
+
+@pytest.mark.parametrize("pool", [(0, 1), (1, 5), (2, 3)])
+def test_fused_importance_topk_equals_the_two_calls_and_the_checker(pool):
+    """pdd_importance_topk: scores and mask bit-identical to pdd_token_importance followed by
+    pdd_refine_topk, and the mask equal to the checker's exact top-k of those scores."""
+    import torch
+    from oracle import pdd_oracle as orc
+    from paper_2508_09035_b200 import binding as B
+    w = wl.small_like("fused", 880, 8, 2, 128, 1500, 512, 40, keep_ratio=0.3, window="all")
+    s = w.seqs[0]
+    kv = H.make_cache(w, 0)
+    for c in s.calls:
+        sl = slice(c.pos0, c.pos0 + c.length)
+        fn = kv.prefill_chunk if c.kind == wl.PROMPT else kv.append_received
+        fn(H.to_dev(s.q[sl]), H.to_dev(s.k[sl]), H.to_dev(s.v[sl]), window=c.window)
+    n = s.n_tokens
+    score2 = kv.token_importance(0, pool[0], pool[1])
+    keep2, n2 = kv.refine_topk(score2, 0.3, 0, 7, n - 5)
+    for with_score in (True,):
+        score1 = torch.full((n,), -1.0, dtype=torch.float32, device="cuda:0")
+        keep1 = torch.full((n,), 9, dtype=torch.uint8, device="cuda:0")
+        n1 = torch.full((1,), -1, dtype=torch.int32, device="cuda:0")
+        B.pdd_importance_topk(kv.h, 0, pool[0], pool[1], score1.data_ptr() if with_score else None,
+                              0, 7, n - 5, 0.3, keep1.data_ptr(), n1.data_ptr(), kv.stream)
+        torch.cuda.synchronize()
+        if with_score:
+            assert torch.equal(score1, score2)
+        assert torch.equal(keep1, keep2) and int(n1.item()) == int(n2.item())
+    want, want_n, _ = orc.refine_topk(score2.cpu().numpy(), s.kind, 7, n - 5, 0.3)
+    np.testing.assert_array_equal(keep2.cpu().numpy(), want)
+    # accumulate adds to the caller's vector, as the separate call does
+    acc1 = score2.clone()
+    acc2 = score2.clone()
+    keep1 = torch.empty(n, dtype=torch.uint8, device="cuda:0")
+    n1 = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    B.pdd_importance_topk(kv.h, 0, pool[0], pool[1], acc1.data_ptr(), 1, 0, n, 0.3,
+                          keep1.data_ptr(), n1.data_ptr(), kv.stream)
+    kv.token_importance(0, pool[0], pool[1], score=acc2, accumulate=True)
+    assert torch.equal(acc1, acc2)
+    keepa, na = kv.refine_topk(acc2, 0.3, 0)
+    assert torch.equal(keep1, keepa) and int(n1.item()) == int(na.item())
+    kv.close()
+
+
+def test_batched_importance_equals_single_calls():
+    import torch
+    from paper_2508_09035_b200 import binding as B
+    w = wl.ragged_batch("imp_b", 881, 8, 2, 64, 5, 100, 900, 256, 30, 0.4, "last", page_tokens=64)
+    kv = H.make_cache(w, 0)
+    res = H.run_library(w, cache=kv)
+    offs = [0]
+    for s in w.seqs:
+        offs.append(offs[-1] + s.n_tokens)
+    score = torch.full((offs[-1],), -1.0, dtype=torch.float32, device="cuda:0")
+    B.pdd_token_importance_batched(kv.h, list(range(len(w.seqs))), 0, 1, score.data_ptr(), offs, 0,
+                                   kv.stream)
+    got = score.cpu().numpy()
+    for si in range(len(w.seqs)):
+        np.testing.assert_array_equal(got[offs[si]:offs[si + 1]], res[si]["score"].astype(np.float32))
+    with pytest.raises(B.PddError):
+        B.pdd_token_importance_batched(kv.h, [0], 0, 1, score.data_ptr(), [0, 3], 0, kv.stream)
+    kv.close()
