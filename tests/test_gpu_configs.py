@@ -94,6 +94,17 @@ def test_config2_full(window):
     # with the checker's, inside it with the exact top-k of the library's own scores.
     print("config2 %s: %s" % (window, stats[0]))
     assert stats[0]["band"] < 2048
+    # Second, tight band: the measured importance error is below 1e-6 relative, so the mask must
+    # also equal the checker's wherever the checker's score is more than 1e-4 (relative) away
+    # from the threshold, and that band must be small enough for the comparison to bite.
+    from oracle import pdd_oracle as orc
+    s = w.seqs[0]
+    score_o = want[0]["score"]
+    keep_o, _, k = orc.refine_topk(score_o, s.kind, 0, s.n_tokens, w.keep_ratio)
+    theta = np.sort(score_o[s.kind == 0])[::-1][k - 1]
+    tight = np.abs(score_o - theta) <= 1e-4 * abs(theta)
+    np.testing.assert_array_equal(got[0]["keep"][~tight], keep_o[~tight])
+    assert int(tight.sum()) <= 64, "tight band holds %d positions" % int(tight.sum())
 
 
 def test_config4_long_prompt_sampled():

@@ -64,6 +64,19 @@ def test_static_buffer_call_matches_two_step_path_twice_in_a_row():
     ref, n_ref, got, n_got = _both_paths(kv2, n2, 0.5, B.PDD_POOL_NONE, 1, 0, n2)
     np.testing.assert_array_equal(got, ref)
     assert n_got == n_ref == 150
+    # the same answer straight from the CPU checker: its importance (fp64 column sums of the
+    # library's own fp32 column sums, no pooling) and its stable-sort top-k; heads are added in
+    # fp32 on the GPU, so positions within that rounding of the threshold may differ
+    from oracle import pdd_oracle as orc
+    cs = kv2.export_colsum(0).cpu().numpy().astype(np.float64)
+    score64 = orc.importance([cs])
+    s2 = w2.seqs[0]
+    want, want_n, k = orc.refine_topk(score64, s2.kind, 0, n2, 0.5)
+    assert n_got == want_n
+    theta = np.sort(score64[s2.kind == 0])[::-1][k - 1]
+    near = np.abs(score64 - theta) <= 1e-6 * abs(theta)
+    np.testing.assert_array_equal(got[~near], want[~near])
+    assert int(near.sum()) <= 4
     # and the first problem again gives the same answer as before
     ref1, n_ref1, got1, n_got1 = _both_paths(kv1, n1, 0.3, B.PDD_POOL_AVG, 7, 100, 1100)
     np.testing.assert_array_equal(got1, ref1)
