@@ -143,6 +143,7 @@ struct Segment {
   int n_kb[2];          // one past the last key block each tile needs (causal extent)
   int nblk[2];          // key blocks of this segment that each tile takes part in
   int rows_valid[2];
+  int seq_pos0;         // cache position of the sequence's first row of this call
   int row0[2];          // packed row of tile row 0
   int p0[2];            // cache position of tile row 0
   int full;             // the segment covers the pair's whole key range
@@ -154,6 +155,7 @@ __device__ __forceinline__ void describe_pair(const CallHeader* hdr, const SeqDe
   sg.w = decode_pair(hdr, descs, pair, g.hq, g.hkv);
   const SeqDesc& sd = descs[sg.w.seq_slot];
   sg.seq_id = sd.seq_id;
+  sg.seq_pos0 = (int)sd.pos0;
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     sg.rows_valid[t] = sg.w.active[t] ? min(kTileRows, sd.len - sg.w.t_local[t] * kTileRows) : 0;
@@ -289,11 +291,14 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
   if (kCluster) ptx::cluster_sync_all();
   const uint32_t tmem = bars->tmem_base;
   volatile int32_t* abort_flag = &bars->abort_flag;
-  // Each role waits for the kernel ahead (its writes: cache rows, page table; its reads: the
-  // buffers this kernel overwrites) at its own point, then looks at the sticky status: a
-  // launch that follows a timed-out wait does no work.
-  auto wait_for_kernels_ahead = [&]() -> bool {
-    ptx::griddep_wait();
+  // When this kernel starts, every kernel before the call's kv_append has completed (kv_append
+  // lets its dependents go only after its own wait), so the only work that may still be in
+  // flight is kv_append's: the call's new cache rows and the page-table entries of their pages.
+  // Nothing else this kernel touches depends on it.  Only the producer therefore waits for the
+  // kernel ahead, and only when it reaches the first key block that holds a new row: key blocks
+  // below pos0 are fetched and multiplied while kv_append is still copying.  A launch that
+  // follows a timed-out wait (sticky status) does no work.
+  auto status_set = [&]() -> bool {
     return *reinterpret_cast<volatile int32_t*>(g.dev_status) != 0;
   };
 
@@ -327,7 +332,8 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
         if (sg.nblk[0] > 0) load_q(std::integral_constant<int, 0>{}, q_cnt0);
         if (sg.nblk[1] > 0) load_q(std::integral_constant<int, 1>{}, q_cnt1);
       }
-      if (wait_for_kernels_ahead()) {
+      bool waited = false;
+      if (status_set()) {
         // nothing to do, but the loads in flight must land before the CTA may exit
         if (q_cnt0 > 0 && !ptx::mbar_wait(&bars->q_full[0], 0)) ok = false;
         if (q_cnt1 > 0 && !ptx::mbar_wait(&bars->q_full[1], 0)) ok = false;
@@ -343,6 +349,10 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
         for (int jj = 0; jj < nmax && ok; ++jj, ++kv_it) {
           const int st = kv_it % kKvStages;
           const uint32_t ph = (uint32_t)(kv_it / kKvStages) & 1;
+          if (!waited && (sg.kb_lo + jj + 1) * kKeyBlock > sg.seq_pos0) {
+            ptx::griddep_wait();           // this block holds rows that kv_append is writing
+            waited = true;
+          }
           int page[2], rin[2];
           for (int hh = 0; hh < 2; ++hh) {
             const int pos = (sg.kb_lo + jj) * kKeyBlock + 64 * hh;
@@ -383,7 +393,7 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
       Segment sg;
       uint32_t kv_it = 0, q_cnt0 = 0, q_cnt1 = 0, n_qk = 0;
       bool ok = true;
-      const bool skip = wait_for_kernels_ahead();
+      const bool skip = status_set();
       auto qk = [&](int t, uint32_t st_k) -> bool {
         if (n_qk > 0 && !ptx::mbar_wait(&bars->s_free, (n_qk - 1) & 1)) return false;
         ++n_qk;
@@ -434,7 +444,7 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
       Segment sg;
       uint32_t kv_it = 0, blk0 = 0, blk1 = 0;
       bool ok = true;
-      const bool skip = wait_for_kernels_ahead();
+      const bool skip = status_set();
       auto pv = [&](int t, uint32_t st_v, bool first, bool last, uint32_t& blk) -> bool {
         if (!ptx::mbar_wait(&bars->p_ready[t], blk & 1)) return false;
         ++blk;
@@ -477,7 +487,7 @@ fwd_attn_kernel(CacheGeom g, const void* __restrict__ rec_global,
     SegmentWalk<kBand, kCluster> walk(rec, cta, csize, crank);
     Segment sg;
     int blk = 0, o_cnt = 0, pv_cnt = 0;
-    bool ok = !wait_for_kernels_ahead();     // (a skipped launch is not a failure: see below)
+    bool ok = !status_set();     // (a skipped launch is not a failure: see below)
     const bool skipped = !ok;
     while (ok && walk.next(g, sg)) {
       const int p_tile = sg.p0[t];
