@@ -405,8 +405,8 @@ def kernel_table(trace, trace_steps: int, w: wl.Workload, peaks) -> dict:
         # read fp32 column sums of every head, write one fp32 score per position
         "importance_reduce": 4 * n_tokens * (w.n_q_heads + 1),
         # scores (fp32) read once into shared memory; kind (1 byte) read by the counting pass,
-        # the four radix passes and the mask pass; the mask pass writes one byte
-        "radix_topk": n_tokens * (4 + 6 + 1),
+        # the three radix passes and the mask pass; the mask pass writes one byte
+        "radix_topk": n_tokens * (4 + 5 + 1),
     }
     out = {}
     for k, (c, ms) in trace.items():

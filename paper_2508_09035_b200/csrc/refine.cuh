@@ -92,6 +92,8 @@ struct TopkSeq {
 };
 
 constexpr int kTopkThreads = 1024;
+constexpr int kRadixBits = 11;                // digits of the radix select
+constexpr int kRadixBins = 1 << kRadixBits;   // = 2 * kTopkThreads: two bins per thread in the scan
 constexpr int kTopkBatch = 64;      // sequences per launch (descriptors travel as parameters)
 struct TopkBatch {
   TopkSeq s[kTopkBatch];
@@ -103,18 +105,18 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// Where the selection keys come from.  ScoreKeys: fp32 scores, 32-bit keys, 4 radix passes.
-// VoteKeys: ready-made 40-bit keys (votes in bits 32-39 above the order key of the summed
-// value), 5 passes.
+// Where the selection keys come from.  ScoreKeys: fp32 scores, 32-bit keys, 3 radix passes of
+// 11 bits.  VoteKeys: ready-made 40-bit keys (votes in bits 32-39 above the order key of the
+// summed value), 4 passes.
 struct ScoreKeys {
   using key_t = uint32_t;
-  static constexpr int kPasses = 4;
+  static constexpr int kPasses = 3;
   const float* score;
   __device__ __forceinline__ key_t load(int64_t i) const { return order_key(score[i]); }
 };
 struct VoteKeys {
   using key_t = unsigned long long;
-  static constexpr int kPasses = 5;
+  static constexpr int kPasses = 4;
   const unsigned long long* key;
   __device__ __forceinline__ key_t load(int64_t i) const { return key[i]; }
 };
@@ -137,7 +139,7 @@ __device__ __forceinline__ void radix_topk_body(const Keys& keys, const uint8_t*
                                                 uint8_t* __restrict__ keep,
                                                 int32_t* __restrict__ n_kept_out) {
   using key_t = typename Keys::key_t;
-  __shared__ int hist[256];
+  __shared__ int hist[kRadixBins];
   __shared__ int warp_buf[kTopkThreads / 32];
   __shared__ key_t s_prefix;
   __shared__ int s_need;
@@ -162,46 +164,49 @@ __device__ __forceinline__ void radix_topk_body(const Keys& keys, const uint8_t*
   kk = kk < 0 ? 0 : (kk > n_cand ? n_cand : kk);
   const int k = (int)kk;
 
-  // Radix select, 8 bits per pass from the top: after the passes s_prefix is the key of
-  // the k-th largest candidate and s_need the number of positions to take at that key.
+  // Radix select, 11 bits per pass from the top (three passes for 32-bit keys): after the
+  // passes s_prefix is the key of the k-th largest candidate and s_need the number of
+  // positions to take at that key.
   if (tid == 0) { s_prefix = 0; s_need = k; }
   __syncthreads();
   if (k > 0) {
     for (int pass = 0; pass < Keys::kPasses; ++pass) {
-      const int shift = 8 * (Keys::kPasses - 1 - pass);
-      const key_t mask_hi = pass == 0 ? (key_t)0 : (key_t)(~(key_t)0 << (shift + 8));
-      for (int b = tid; b < 256; b += kTopkThreads) hist[b] = 0;
+      const int shift = kRadixBits * (Keys::kPasses - 1 - pass);
+      const key_t mask_hi = pass == 0 ? (key_t)0 : (key_t)(~(key_t)0 << (shift + kRadixBits));
+      for (int b = tid; b < kRadixBins; b += kTopkThreads) hist[b] = 0;
       __syncthreads();
       const key_t prefix = s_prefix;
       for (int64_t i = tid; i < sq.n; i += kTopkThreads) {
         const bool cand = (!kd || kd[i] == 0) && i >= sq.cand_lo && i < sq.cand_hi;
         if (!cand) continue;
         const key_t key = keys.load(sq.offset + i);
-        if ((key & mask_hi) == prefix) atomicAdd(&hist[(int)((key >> shift) & 255)], 1);
+        if ((key & mask_hi) == prefix)
+          atomicAdd(&hist[(int)((key >> shift) & (key_t)(kRadixBins - 1))], 1);
       }
       __syncthreads();
-      // The bin that holds the need-th largest key: thread i < 256 looks at bin 255 - i, so an
-      // inclusive scan over threads is the count of keys in that bin and all higher bins.
+      // The bin that holds the need-th largest key: thread i looks at bins B-1-2i and B-2-2i,
+      // so an inclusive scan of the pair sums over threads is the count of keys in those bins
+      // and all higher ones.
       const int need = s_need;
       __syncthreads();                         // everyone has read s_need before it changes
-      int v = 0, incl = 0;
-      if (tid < 256) {
-        v = hist[255 - tid];
-        incl = v;
-        for (int off = 1; off < 32; off <<= 1) {
-          const int up = __shfl_up_sync(0xffffffffu, incl, off);
-          if ((tid & 31) >= off) incl += up;
-        }
-        if ((tid & 31) == 31) warp_buf[tid >> 5] = incl;
+      const int bin_a = kRadixBins - 1 - 2 * tid, bin_b = bin_a - 1;
+      const int va = hist[bin_a], vb = hist[bin_b];
+      int incl = va + vb;
+      for (int off = 1; off < 32; off <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, off);
+        if ((tid & 31) >= off) incl += up;
       }
+      if ((tid & 31) == 31) warp_buf[tid >> 5] = incl;
       __syncthreads();
-      if (tid < 256) {
-        for (int w = 0; w < (tid >> 5); ++w) incl += warp_buf[w];
-        // exactly one bin satisfies this (the total count of matching keys is >= need)
-        if (incl >= need && incl - v < need) {
-          s_prefix = prefix | ((key_t)(255 - tid) << shift);
-          s_need = need - (incl - v);
-        }
+      for (int w = 0; w < (tid >> 5); ++w) incl += warp_buf[w];
+      const int excl = incl - (va + vb);
+      // exactly one bin satisfies this (the total count of matching keys is >= need)
+      if (excl < need && excl + va >= need) {
+        s_prefix = prefix | ((key_t)bin_a << shift);
+        s_need = need - excl;
+      } else if (excl + va < need && incl >= need) {
+        s_prefix = prefix | ((key_t)bin_b << shift);
+        s_need = need - (excl + va);
       }
       __syncthreads();
     }
@@ -264,14 +269,14 @@ radix_topk_kernel(const Keys keys, const uint8_t* __restrict__ kinds,
 // Keys held in shared memory (filled by the fused kernel below): read from global memory once.
 struct SmemScoreKeys {
   using key_t = uint32_t;
-  static constexpr int kPasses = 4;
+  static constexpr int kPasses = 3;
   const uint32_t* key;
   __device__ __forceinline__ key_t load(int64_t i) const { return key[i]; }
 };
 
 // Selection with the keys staged in shared memory: a CTA reads its sequence's scores from
 // global memory once (n * 4 bytes of dynamic shared memory, at most kStagedTopkMax positions per
-// sequence) and the four radix passes and the mask pass work on the staged keys.
+// sequence) and the radix passes and the mask pass work on the staged keys.
 constexpr int64_t kStagedTopkMax = 49152;       // positions (192 KiB of keys)
 __global__ void __launch_bounds__(kTopkThreads)
 radix_topk_staged_kernel(const float* __restrict__ score, const uint8_t* __restrict__ kinds,
