@@ -468,7 +468,8 @@ def run_reference(args, rank: int, world: int):
                 n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
                 ms_per_step=1e3 * t_total / args.steps, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload=w.name, description=w.description, window=args.window),
+                config=dict(workload=w.name, description=w.description, window=args.window,
+                            keep_ratio=w.keep_ratio, passes_per_step=1, parallelism="1 gpu"),
                 cpu_baseline=dict(value=value, unit="tokens/s", cores=cores, kind="oracle",
                                   sample=sample),
                 e2e=dict(value=value, unit="tokens/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
