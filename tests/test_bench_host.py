@@ -87,3 +87,29 @@ def test_grouped_calls_cover_every_call_once():
         assert seen[si] == [c.pos0 for c in s.calls]
     w2 = wl.config_c2()
     assert [g[0][1].pos0 for _, _, g in bench.grouped_calls(w2)] == [c.pos0 for c in w2.seqs[0].calls]
+
+
+def test_attention_bytes_per_launch_and_traffic_scaling():
+    """Algorithmic bytes of the mean attention launch: q + out of the call's rows and one read of
+    the sequence's K and V up to its new length; the ncu capture is scaled by that figure and is
+    dropped when the kernel source no longer matches the capture."""
+    w = wl.small_like("bytes", 3, 8, 2, 128, 512, 256, 0, window="last")
+    # two calls of 256 rows: lengths 256 and 512 after them
+    per_row_q = 8 * 128 * 2
+    per_pos_kv = 2 * 2 * 128 * 2
+    want = (2 * 256 * per_row_q + 256 * per_pos_kv + 2 * 256 * per_row_q + 512 * per_pos_kv) / 2
+    assert bench.attention_bytes_per_launch(w) == want
+    cap = dict(bench.FWD_ATTN_TRAFFIC_CAPTURE)
+    try:
+        bench.FWD_ATTN_TRAFFIC_CAPTURE.update(dram_bytes=2.0e6, algorithmic_bytes=1.0e6,
+                                              source_sha256=bench.attention_source_tag())
+        assert bench.scaled_traffic(w) == 2.0 * want
+        bench.FWD_ATTN_TRAFFIC_CAPTURE.update(source_sha256="not the kernel's hash")
+        assert bench.scaled_traffic(w) is None
+    finally:
+        bench.FWD_ATTN_TRAFFIC_CAPTURE.update(cap)
+
+
+def test_traffic_capture_belongs_to_the_kernel_source_in_the_tree():
+    """The committed capture must have been taken on the committed attention kernel."""
+    assert bench.FWD_ATTN_TRAFFIC_CAPTURE["source_sha256"] == bench.attention_source_tag()
