@@ -47,8 +47,8 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # one read of the sequence's K and V per call), so `roofline.traffic` scales the capture to the
 # mean launch of the timed workload.  The capture belongs to one version of the kernel source:
 # if csrc/attn_tc.cuh has changed since (first 12 hex digits of its sha256), traffic is null.
-FWD_ATTN_TRAFFIC_CAPTURE = dict(dram_bytes=70.467e6, algorithmic_bytes=67.109e6,
-                                source_sha256="be500b1b82f0")
+FWD_ATTN_TRAFFIC_CAPTURE = dict(dram_bytes=69.590e6, algorithmic_bytes=67.109e6,
+                                source_sha256="65d70472c945")
 TARGET_TIMED_MS = 120.0          # a timed region at least this long (>= 20 clock samples at 4 ms)
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0

@@ -851,46 +851,55 @@ attn_combine_kernel(CacheGeom g, const void* __restrict__ rec, __nv_bfloat16* __
   // Segments are taken four at a time with every load issued before its use and no branch
   // around a load (an empty segment gets weight 0; its slot holds finite stale values), so
   // that the L2 round trips of the segments overlap instead of adding up.
+  // (two at a time when the pair has only two segments, by far the most common case: no slot
+  // is then read twice)
   float M = -INFINITY;
-  for (int s0 = 0; s0 < sp.n_seg; s0 += 4) {
-    float2 ml[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      ml[u] = g.part_ml[slot_of(min(s0 + u, sp.n_seg - 1)) * part_ml_elems() + t * 128 + r];
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (ml[u].y > 0.f) M = fmaxf(M, ml[u].x);
-  }
   float Lsum = 0.f;
   float acc[32];
 #pragma unroll
   for (int c = 0; c < 32; ++c) acc[c] = 0.f;
-  for (int s0 = 0; s0 < sp.n_seg; s0 += 4) {
-    float2 ml[4];
-    float4 v[4][8];
+  auto merge = [&](auto width) {
+    constexpr int U = decltype(width)::value;
+    for (int s0 = 0; s0 < sp.n_seg; s0 += U) {
+      float2 ml[U];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const size_t slot = slot_of(min(s0 + u, sp.n_seg - 1));
-      ml[u] = g.part_ml[slot * part_ml_elems() + t * 128 + r];
-      const float4* po = reinterpret_cast<const float4*>(g.part_o + slot * part_o_floats(D)) +
-                         ((size_t)t * (D / 4) + cg * 8) * 128 + r;
+      for (int u = 0; u < U; ++u)
+        ml[u] = g.part_ml[slot_of(min(s0 + u, sp.n_seg - 1)) * part_ml_elems() + t * 128 + r];
 #pragma unroll
-      for (int c4 = 0; c4 < 8; ++c4) v[u][c4] = po[(size_t)c4 * 128];
+      for (int u = 0; u < U; ++u)
+        if (ml[u].y > 0.f) M = fmaxf(M, ml[u].x);
     }
+    for (int s0 = 0; s0 < sp.n_seg; s0 += U) {
+      float2 ml[U];
+      float4 v[U][8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const bool live = s0 + u < sp.n_seg && ml[u].y > 0.f;
-      const float wgt = live ? ptx::ex2((ml[u].x - M) * sl2) : 0.f;
-      Lsum = fmaf(wgt, live ? ml[u].y : 0.f, Lsum);
+      for (int u = 0; u < U; ++u) {
+        const size_t slot = slot_of(min(s0 + u, sp.n_seg - 1));
+        ml[u] = g.part_ml[slot * part_ml_elems() + t * 128 + r];
+        const float4* po = reinterpret_cast<const float4*>(g.part_o + slot * part_o_floats(D)) +
+                           ((size_t)t * (D / 4) + cg * 8) * 128 + r;
 #pragma unroll
-      for (int c4 = 0; c4 < 8; ++c4) {
-        acc[4 * c4 + 0] = fmaf(wgt, v[u][c4].x, acc[4 * c4 + 0]);
-        acc[4 * c4 + 1] = fmaf(wgt, v[u][c4].y, acc[4 * c4 + 1]);
-        acc[4 * c4 + 2] = fmaf(wgt, v[u][c4].z, acc[4 * c4 + 2]);
-        acc[4 * c4 + 3] = fmaf(wgt, v[u][c4].w, acc[4 * c4 + 3]);
+        for (int c4 = 0; c4 < 8; ++c4) v[u][c4] = po[(size_t)c4 * 128];
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const bool live = s0 + u < sp.n_seg && ml[u].y > 0.f;
+        const float wgt = live ? ptx::ex2((ml[u].x - M) * sl2) : 0.f;
+        Lsum = fmaf(wgt, live ? ml[u].y : 0.f, Lsum);
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+          acc[4 * c4 + 0] = fmaf(wgt, v[u][c4].x, acc[4 * c4 + 0]);
+          acc[4 * c4 + 1] = fmaf(wgt, v[u][c4].y, acc[4 * c4 + 1]);
+          acc[4 * c4 + 2] = fmaf(wgt, v[u][c4].z, acc[4 * c4 + 2]);
+          acc[4 * c4 + 3] = fmaf(wgt, v[u][c4].w, acc[4 * c4 + 3]);
+        }
       }
     }
-  }
+  };
+  if (sp.n_seg <= 2)
+    merge(std::integral_constant<int, 2>{});
+  else
+    merge(std::integral_constant<int, 4>{});
   const float inv = 1.f / Lsum;
   __nv_bfloat16* orow =
       out + ((size_t)(sg.row0[t] + r) * g.hq + sg.w.head[t]) * D + cg * 32;
