@@ -13,14 +13,19 @@
 // this is a second score pass that reads the LSE the attention kernel wrote.
 //   warp 0    TMA producer (K tile once, Q tiles through a 2-stage ring)
 //   warp 1    MMA issuer; two 128-column accumulators in TMEM alternate
-//   warps 2-5 consumers
+//   warps 2-5 consumers of the even items (accumulator 0), warps 6-9 of the odd items
+//             (accumulator 1): with two CTAs per SM four consumer warps share a scheduler,
+//             which is what keeps the MUFU unit busy (two left it idle half of the time)
+// A head's items go to both consumer groups, so each group leaves its partial sum of a
+// (head, key) in shared memory and one thread adds the two in a fixed order at the end.
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
 
 namespace pdd {
 
-constexpr int kColsumThreads = 192;
+constexpr int kColsumThreads = 320;
+constexpr int kColsumMaxHeads = 8;      // query heads per CTA (more are dealt out to further CTAs)
 // Pairs of every 4 whose exp2 is a polynomial on the FMA pipe (measured on the long-prompt
 // window pass: 0 -> 0.83 ms, 1 -> 0.78, 2 -> 0.80, 3 -> 0.91).
 constexpr int kColsumPoly = 1;
@@ -38,8 +43,9 @@ struct ColsumSmem {
   static constexpr int kTileBytes = kSub * kSubBytes;
   static constexpr int kKOff = 0;
   static constexpr int kQOff = kTileBytes;                 // 2 stages
-  static constexpr int kLseOff = 3 * kTileBytes;           // 2 x 128 floats
-  static constexpr int kBarOff = kLseOff + 1024;
+  static constexpr int kLseOff = 3 * kTileBytes;           // 2 groups x 2 buffers x 128 floats
+  static constexpr int kPartOff = kLseOff + 2048;          // 2 groups x kColsumMaxHeads x 128 floats
+  static constexpr int kBarOff = kPartOff + 2 * kColsumMaxHeads * 512;
   static constexpr int kBytes = kBarOff + 256 + 1024;
 };
 
@@ -64,6 +70,7 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
   uint8_t* sK = base + L::kKOff;
   uint8_t* sQ = base + L::kQOff;
   float* sLse = reinterpret_cast<float*>(base + L::kLseOff);
+  float* sPart = reinterpret_cast<float*>(base + L::kPartOff);
   ColsumBars* bars = reinterpret_cast<ColsumBars*>(base + L::kBarOff);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -120,6 +127,7 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
     bars->abort_flag = 0;
     ptx::fence_mbar_init();
   }
+  for (int i = tid; i < 2 * kColsumMaxHeads * 128; i += kColsumThreads) sPart[i] = 0.f;
   if (warp == 1) {
     ptx::tmem_alloc(&bars->tmem_base, 256);
     ptx::tmem_relinquish();
@@ -187,15 +195,16 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
       if (!ok) *abort_flag = 1;
     }
   } else {
+    const int cg = (warp - 2) >> 2;                   // consumer group: items cg, cg + 2, ...
     const int wq = warp & 3;                          // TMEM lane quarter this warp may read
     const int r = wq * 32 + lane;                     // key row of the tile
-    const int ct = tid - 64;                          // 0..127 among the consumers
+    const int ct = (tid - 64) & 127;                  // 0..127 inside the group
     const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
     const int64_t key = key0 + r;
     const float sl2 = g.scale * 1.4426950408889634f;
     float acc = 0.f;
-    int cur_h = h_first;
     bool ok = true;
+    float* const part = sPart + (size_t)cg * kColsumMaxHeads * 128 + r;    // [head of the CTA][key]
     // LSE (exp2 domain) of the rows of an item's query tile; fetched one item ahead so that the
     // global-memory latency falls under the previous item's exponentials.
     auto fetch_lse = [&](int h, int qt) -> float {
@@ -204,30 +213,35 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
       return ct < rows_valid ? g.lse[(size_t)h * g.lse_ld + row0 + ct] * 1.4426950408889634f : 0.f;
     };
     // item it = (head h_first + it / n_qt_act, query tile qt_min + it % n_qt_act), stepped
-    // without divisions; (hn, qn) is the item after it
-    int h = h_first, qt = qt_min, hn = h_first, qn = qt_min;
-    float lse_next = fetch_lse(h, qt);
-    for (int it = 0; it < n_items; ++it, h = hn, qt = qn) {
-      const int st = it & 1;
-      const uint32_t ph = (uint32_t)(it >> 1) & 1;
-      qn = qt + 1;
-      hn = h;
-      if (qn == qt_end) {
-        qn = qt_min;
-        ++hn;
+    // without divisions; this group takes items cg, cg + 2, ...; (hn, qn) is its next item
+    auto advance = [&](int& hh, int& qq) {
+      if (++qq == qt_end) {
+        qq = qt_min;
+        ++hh;
       }
+    };
+    int h = h_first, qt = qt_min;
+    if (cg) advance(h, qt);
+    int hn = h, qn = qt, cur_h = h;
+    float lse_next = cg < n_items ? fetch_lse(h, qt) : 0.f;
+    for (int it = cg, n = 0; it < n_items; it += 2, ++n, h = hn, qt = qn) {
+      const int st = cg;                          // the group's accumulator and Q stage
+      const uint32_t ph = (uint32_t)n & 1;
+      advance(hn, qn);
+      advance(hn, qn);
       if (h != cur_h) {
-        if (key < T) g.colsum[((size_t)sd.seq_id * g.hq + cur_h) * g.max_tokens_per_seq + key] += acc;
+        part[(cur_h - h_first) * 128] = acc;
         acc = 0.f;
         cur_h = h;
       }
       const int rows_valid = min(kTileRows, sd.len - qt * kTileRows);
       const int64_t pq0 = sd.pos0 + (int64_t)qt * kTileRows;     // position of query column 0
-      // (the stage's previous reader, item it-2, finished before this thread arrived on
-      // s_empty for it, and every thread's arrival precedes the MMA that precedes s_full)
-      sLse[st * 128 + ct] = lse_next;
+      // (two LSE buffers per group: a thread that is already at item n + 1 writes the other one
+      // than the threads still reading item n)
+      float* const lse_buf = sLse + (cg * 2 + (n & 1)) * 128;
+      lse_buf[ct] = lse_next;
       ptx::mbar_arrive(&bars->lse_ready[st]);
-      if (it + 1 < n_items) lse_next = fetch_lse(hn, qn);
+      if (it + 2 < n_items) lse_next = fetch_lse(hn, qn);
       ok = ptx::mbar_wait(&bars->lse_ready[st], ph);
       if (ok) ok = ptx::mbar_wait(&bars->s_full[st], ph);
       ok = __all_sync(0xffffffffu, ok);
@@ -235,28 +249,27 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
       ptx::tc_fence_after();
       const bool full = rows_valid == kTileRows && pq0 >= key0 + kKeyBlock - 1 &&
                         pq0 + kTileRows - 1 - key0 < g.window;
-      // LSE of the 32 columns in hand, as eight 16-byte shared-memory loads (every thread of
+      // LSE of the 16 columns in hand, as four 16-byte shared-memory loads (every thread of
       // the warp reads the same words: one broadcast each).  Going through the generic float
       // pointer instead costs one load instruction per exponential, and those loads, not the
       // MUFU unit, then bound the kernel.
-      const uint32_t ls_addr = ptx::smem_u32(sLse + st * 128);
-      // 32 query columns at a time; the next 32 are on their way while these are
+      const uint32_t ls_addr = ptx::smem_u32(lse_buf);
+      // 16 query columns at a time; the next 16 are on their way while these are
       // exponentiated, and the accumulator goes back to the MMA thread as soon as the last
       // ones have landed in registers.  Two partial sums, added in a fixed order.
       float acc0 = 0.f, acc1 = 0.f;
-      auto add32 = [&](int c4, const uint32_t* v) {
-        float ls[32];
+      auto add16 = [&](int c16, const uint32_t* v) {
+        float ls[16];
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < 4; ++i)
           asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
                        : "=f"(ls[4 * i]), "=f"(ls[4 * i + 1]), "=f"(ls[4 * i + 2]), "=f"(ls[4 * i + 3])
-                       : "r"(ls_addr + (uint32_t)(c4 * 128 + i * 16)));
+                       : "r"(ls_addr + (uint32_t)(c16 * 64 + i * 16)));
         if (full) {
-          // The MUFU unit (16 exponentials per clock per SM) bounds this loop, so kColsumPoly
-          // of every 4 pairs go through a cubic on the FMA pipe instead (7.5e-5 relative
-          // error against a 1e-2 bound on the sums).
+          // kColsumPoly of every 4 pairs go through a cubic on the FMA pipe instead of the MUFU
+          // unit (7.5e-5 relative error against a 1e-2 bound on the sums).
 #pragma unroll
-          for (int c = 0; c < 32; c += 8) {
+          for (int c = 0; c < 16; c += 8) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const float x0 = fmaf(__uint_as_float(v[c + 2 * i]), sl2, -ls[c + 2 * i]);
@@ -273,8 +286,8 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
           }
         } else {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const int col = c4 * 32 + c;
+          for (int c = 0; c < 16; ++c) {
+            const int col = c16 * 16 + c;
             const float e = ex2f_cs(fmaf(__uint_as_float(v[c]), sl2, -ls[c]));
             const float ee = (col < rows_valid && pq0 + col >= key && pq0 + col - key < g.window) ? e : 0.f;
             if (c & 1) acc1 += ee; else acc0 += ee;
@@ -282,26 +295,35 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
         }
       };
       const uint32_t tacc = tmem + 128 * st + lane_base;
-      uint32_t va[32], vb[32];
-      ptx::tmem_ld32(tacc, va);
-      ptx::tmem_ld_wait();
-      ptx::tmem_ld32(tacc + 32, vb);
-      add32(0, va);
-      ptx::tmem_ld_wait();
-      ptx::tmem_ld32(tacc + 64, va);
-      add32(1, vb);
-      ptx::tmem_ld_wait();
-      ptx::tmem_ld32(tacc + 96, vb);
-      add32(2, va);
-      ptx::tmem_ld_wait();
-      ptx::tc_fence_before();
-      ptx::mbar_arrive(&bars->s_empty[st]);
-      add32(3, vb);
+      uint32_t va[16], vb[16];
+      ptx::tmem_ld16(tacc, va);
+#pragma unroll
+      for (int c16 = 0; c16 < 8; c16 += 2) {
+        ptx::tmem_ld_wait();
+        ptx::tmem_ld16(tacc + 16 * (c16 + 1), vb);
+        add16(c16, va);
+        ptx::tmem_ld_wait();
+        if (c16 + 2 < 8) {
+          ptx::tmem_ld16(tacc + 16 * (c16 + 2), va);
+        } else {
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(&bars->s_empty[st]);
+        }
+        add16(c16 + 1, vb);
+      }
       acc += acc0 + acc1;
     }
-    if (ok && key < T)
-      g.colsum[((size_t)sd.seq_id * g.hq + cur_h) * g.max_tokens_per_seq + key] += acc;
+    if (cg < n_items) part[(cur_h - h_first) * 128] = acc;
     if (!ok && lane == 0) *abort_flag = 1;
+    // Both groups' partial sums stand: the threads of group cg finish heads cg, cg + 2, ... of
+    // the CTA, each the only writer of its (head, key) in global memory.
+    ptx::named_bar_sync(1, 256);
+    if (!*abort_flag && key < T) {
+      for (int hl = cg; hl < hpc; hl += 2) {
+        const float sum = sPart[hl * 128 + r] + sPart[(kColsumMaxHeads + hl) * 128 + r];
+        g.colsum[((size_t)sd.seq_id * g.hq + h_first + hl) * g.max_tokens_per_seq + key] += sum;
+      }
+    }
   }
 
   ptx::tc_fence_before();
@@ -334,7 +356,8 @@ inline cudaError_t launch_colsum_tc(const CacheGeom& g, const void* rec_dev, int
   // still fits one wave (the K tile is then fetched once per part, from L2).
   const int G = g.hq / g.hkv, slots = 2 * sm_count;
   int hsplit = 1;
-  for (int s = 2; s <= G; ++s)
+  while (G % hsplit != 0 || G / hsplit > kColsumMaxHeads) ++hsplit;     // ends at G at the latest
+  for (int s = hsplit + 1; s <= G; ++s)
     if (G % s == 0 && (int64_t)n_kb_total * g.hkv * s <= slots) hsplit = s;
   dim3 grid((unsigned)n_kb_total, (unsigned)(g.hkv * hsplit));
   if (g.d == 128)
