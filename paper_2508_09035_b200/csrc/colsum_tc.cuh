@@ -202,15 +202,16 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
     const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
     const int64_t key = key0 + r;
     const float sl2 = g.scale * 1.4426950408889634f;
+    const float2 sl2v = make_float2(sl2, sl2);
     float acc = 0.f;
     bool ok = true;
     float* const part = sPart + (size_t)cg * kColsumMaxHeads * 128 + r;    // [head of the CTA][key]
-    // LSE (exp2 domain) of the rows of an item's query tile; fetched one item ahead so that the
-    // global-memory latency falls under the previous item's exponentials.
+    // Minus the LSE (exp2 domain) of the rows of an item's query tile; fetched one item ahead so
+    // that the global-memory latency falls under the previous item's exponentials.
     auto fetch_lse = [&](int h, int qt) -> float {
       const int rows_valid = min(kTileRows, sd.len - qt * kTileRows);
       const int64_t row0 = sd.tok_offset + (int64_t)qt * kTileRows;
-      return ct < rows_valid ? g.lse[(size_t)h * g.lse_ld + row0 + ct] * 1.4426950408889634f : 0.f;
+      return ct < rows_valid ? g.lse[(size_t)h * g.lse_ld + row0 + ct] * -1.4426950408889634f : 0.f;
     };
     // item it = (head h_first + it / n_qt_act, query tile qt_min + it % n_qt_act), stepped
     // without divisions; this group takes items cg, cg + 2, ...; (hn, qn) is its next item
@@ -268,27 +269,27 @@ colsum_tc_kernel(CacheGeom g, const void* __restrict__ rec, int hsplit,
         if (full) {
           // kColsumPoly of every 4 pairs go through a cubic on the FMA pipe instead of the MUFU
           // unit (7.5e-5 relative error against a 1e-2 bound on the sums).
+          // (packed fp32x2 multiply-add and add: the issue slots, 60 % busy, are the next bound)
+          float2 a01 = make_float2(acc0, acc1);
 #pragma unroll
           for (int c = 0; c < 16; c += 8) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              const float x0 = fmaf(__uint_as_float(v[c + 2 * i]), sl2, -ls[c + 2 * i]);
-              const float x1 = fmaf(__uint_as_float(v[c + 2 * i + 1]), sl2, -ls[c + 2 * i + 1]);
-              if (i < kColsumPoly) {
-                const float2 e = ptx::ex2_poly2(make_float2(x0, x1));
-                acc0 += e.x;
-                acc1 += e.y;
-              } else {
-                acc0 += ex2f_cs(x0);
-                acc1 += ex2f_cs(x1);
-              }
+              const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[c + 2 * i]),
+                                                      __uint_as_float(v[c + 2 * i + 1])),
+                                          sl2v, make_float2(ls[c + 2 * i], ls[c + 2 * i + 1]));
+              const float2 e = i < kColsumPoly ? ptx::ex2_poly2(x)
+                                               : make_float2(ex2f_cs(x.x), ex2f_cs(x.y));
+              a01 = __fadd2_rn(a01, e);
             }
           }
+          acc0 = a01.x;
+          acc1 = a01.y;
         } else {
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
             const int col = c16 * 16 + c;
-            const float e = ex2f_cs(fmaf(__uint_as_float(v[c]), sl2, -ls[c]));
+            const float e = ex2f_cs(fmaf(__uint_as_float(v[c]), sl2, ls[c]));
             const float ee = (col < rows_valid && pq0 + col >= key && pq0 + col - key < g.window) ? e : 0.f;
             if (c & 1) acc1 += ee; else acc0 += ee;
           }
