@@ -926,7 +926,7 @@ int pdd_refine_topk_batched(const float* score, const uint8_t* kinds, int32_t n_
     if (dev >= 0 && dev < kMaxDevices && !attr_set[dev]) {
       PDD_CUDA(cudaFuncSetAttribute(radix_topk_staged_kernel,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)(kStagedTopkMax * 4)));
+                                    (int)staged_topk_smem_bytes(kStagedTopkMax)));
       attr_set[dev] = true;
     }
   }
@@ -942,7 +942,7 @@ int pdd_refine_topk_batched(const float* score, const uint8_t* kinds, int32_t n_
     }
     if (staged)
       PDD_CUDA(launch_pdl(radix_topk_staged_kernel, dim3(cnt), dim3(kTopkThreads),
-                          (size_t)std::max<int64_t>(n_max, 1) * 4, st, score, kinds, tb, keep_ratio,
+                          staged_topk_smem_bytes(std::max<int64_t>(n_max, 1)), st, score, kinds, tb, keep_ratio,
                           keep, n_kept + base));
     else
       PDD_CUDA(launch_pdl(radix_topk_kernel<ScoreKeys>, dim3(cnt), dim3(kTopkThreads), 0, st,
