@@ -60,3 +60,16 @@ def test_random_ragged_batch(i):
     got = H.run_library(w, cache=kv)
     kv.close()
     H.compare_full(w, got, H.oracle_full(w), what="batch %d" % i)
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(11, 1, 128), (12, 1, 64), (16, 1, 128), (32, 2, 128), (40, 2, 64)])
+def test_large_gqa_groups(hq, hkv, d):
+    """Groups of more than eight query heads: the column-sum kernel keeps at most eight heads'
+    partial sums per CTA and deals the rest out to further CTAs (a prime group size leaves one
+    head per CTA)."""
+    w = wl.small_like("gqa%d_%d" % (hq, hkv), 9900 + hq, hq, hkv, d, 520, 200, 24, keep_ratio=0.4,
+                      window="all", page_tokens=64)
+    kv = H.make_cache(w, 0)
+    got = H.run_library(w, cache=kv)
+    kv.close()
+    H.compare_full(w, got, H.oracle_full(w), what="hq %d hkv %d d %d" % (hq, hkv, d))
