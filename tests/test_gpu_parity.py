@@ -220,7 +220,7 @@ def test_radix_topk_bit_exact_against_sort():
     from paper_2508_09035_b200 import binding as B
     orc = _orc()
     rng = wl.rng_for(170)
-    for n in [1, 2, 31, 32, 33, 1000, 1024, 1025, 4160, 33024, 70001]:
+    for n in [1, 2, 31, 32, 33, 1000, 1024, 1025, 4160, 8191, 33024, 49151, 49152, 49153, 70001]:
         for rep in range(3):
             score, kind, lo, hi, r = _topk_case(rng, n)
             d_score = torch.from_numpy(score).cuda()
