@@ -630,7 +630,7 @@ class StackRunner:
 
 
 def measure(name: str, window: str, steps: int, warmup: int, device, local: int, peaks,
-            world: int = 1, barrier=None) -> dict:
+            world: int = 1, barrier=None, schedule: int = 0) -> dict:
     """Times one workload: HBM-resident passes, end-to-end passes, then a traced pass for the
     per-kernel figures.  Returns the fields of a bench line (or of an `also` entry)."""
     import torch
@@ -646,6 +646,8 @@ def measure(name: str, window: str, steps: int, warmup: int, device, local: int,
     else:
         w = get_workload(name, window)
         runner = Runner(w, device)
+        if schedule:
+            runner.kv.set_schedule(schedule)     # pins one way of cutting the attention work
         tokens, wname, description = w.n_tokens, w.name, w.description
         keep_ratio, flops = w.keep_ratio, w.attention_flops()
     barrier = barrier or (lambda: torch.cuda.synchronize(device))
@@ -754,6 +756,8 @@ def main():
     ap.add_argument("--cpu-baseline-stride", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-also", action="store_true")
+    ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2, 3, 4],
+                    help="pin how the attention kernel's work is cut (0: the library's cost model)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -778,7 +782,7 @@ def main():
         torch.cuda.synchronize(device)
 
     m = measure(args.workload, args.window, args.steps, args.warmup, device, local, peaks, world,
-                barrier)
+                barrier, args.schedule)
     also = []
     if not args.no_also and world == 1:
         for name, k in ALSO_WORKLOADS:
@@ -809,7 +813,8 @@ def main():
                     e2e_copies="pinned host -> device per call on a copy stream, overlapped with "
                                "the previous call's kernels; keep mask read back; the attention "
                                "output stays on the device (the next layer reads it there)",
-                    parallelism="replicas only" if world > 1 else "1 gpu", n_kept=m["n_kept"]),
+                    parallelism="replicas only" if world > 1 else "1 gpu", n_kept=m["n_kept"],
+                    **({"attention_schedule": args.schedule} if args.schedule else {})),
         attention_tflops=m["attention_tflops"],
         attention_tflops_with_combine=m["attention_tflops_with_combine"],
         attention_frac_of_nominal_peak=m["frac_of_nominal_peak"],

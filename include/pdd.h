@@ -363,9 +363,13 @@ int pdd_set_kernel_path(pdd_kv* kv, int32_t path);
  * (tile pair, key block) units, partial results merged by a second kernel; 3 = a
  * thread-block cluster per tile pair whose CTAs split the pair's key range and merge
  * through distributed shared memory (falls back to the cost model for a call whose pairs
- * do not fit on the device at once).  Results are the same up to rounding; 1-3 exist so
- * that tests can pin each one.  The paper has no counterpart (it leaves the attention
- * kernel to the vendor library, Sec. 3.2). */
+ * do not fit on the device at once); 4 = the pair-of-CTAs kernel: clusters of two CTAs work
+ * on four query tiles of one GQA group at a time, every MMA issued once for both CTAs, each
+ * CTA holding half of every K and V block (head_dim 128, no sliding window, group size a
+ * multiple of 4; any other call is cut as under 0).  The cost model never picks 4: on B200
+ * it is the slower kernel, kept so that the comparison can be repeated.  Results are the
+ * same up to rounding; 1-4 exist so that tests can pin each one.  The paper has no
+ * counterpart (it leaves the attention kernel to the vendor library, Sec. 3.2). */
 int pdd_set_schedule(pdd_kv* kv, int32_t mode);
 
 const char* pdd_strerror(int status);

@@ -45,7 +45,10 @@ struct CallHeader {
   // the CtaStart / SplitPair tables are not used (n_ctas = n_pairs * cluster).
   int32_t cluster;
   int32_t rec_bytes;   // size of the whole record (header, descriptors, page ids, schedule)
-  int32_t pad[2];
+  // 1: the launch is the pair-of-CTAs kernel (clusters of two; the CtaStart table then counts
+  // quads, i.e. pairs 2i and 2i+1, and has n_ctas / 2 + 1 entries)
+  int32_t pair_of_ctas;
+  int32_t pad;
 };
 
 // First unit of a CTA's share: key block `kb` of pair `pair`; entry n_ctas is the end.

@@ -16,6 +16,7 @@
 #include "../../include/pdd.h"
 #include "attn_simt.cuh"
 #include "attn_tc.cuh"
+#include "attn_tc2.cuh"
 #include "attn_tc_v0.cuh"
 #include "colsum_tc.cuh"
 #include "common.cuh"
@@ -119,8 +120,9 @@ struct pdd_kv {
   int ring_next;
   CUtensorMap tmK, tmV;
   int kernel_path;
-  int schedule;                       // 0 cost model, 1 whole pairs, 2 equal shares, 3 clusters
+  int schedule;                       // 0 cost model, 1 whole pairs, 2 equal shares, 3 clusters, 4 CTA pairs
   int max_clusters[kMaxCluster + 1];  // clusters of c CTAs the device runs at once
+  int max_clusters2 = 0;              // CTA pairs of the pair-of-CTAs kernel the device runs at once
   int sm_count;
   bool trace;
   std::vector<TraceEntry> trace_log;
@@ -294,8 +296,10 @@ int launch_attention(pdd_kv* kv, const void* rec_dev, const RecParam& recp, int 
   cudaError_t e;
   {
     Tracer t(kv, st, "fwd_attn");
-    e = launch_attn_tc(g, rec_dev, recp, rec_in_param, hdr, tmQ, kv->tmK, kv->tmV,
-                       (__nv_bfloat16*)out, st);
+    e = hdr.pair_of_ctas ? launch_attn_tc2(g, rec_dev, recp, rec_in_param, hdr, tmQ, kv->tmK,
+                                           kv->tmV, (__nv_bfloat16*)out, st)
+                         : launch_attn_tc(g, rec_dev, recp, rec_in_param, hdr, tmQ, kv->tmK, kv->tmV,
+                                          (__nv_bfloat16*)out, st);
   }
   if (e == cudaSuccess && hdr.n_split > 0) {
     Tracer t(kv, st, "attn_combine");
@@ -532,8 +536,14 @@ int run_call(pdd_kv* kv, const pdd_batch* b, const void* q, const void* k, const
     if (kv->schedule == 1) est_b = est_c = 1e30;
     if (kv->schedule == 2) est_a = est_c = 1e30;
     if (kv->schedule == 3 && best_c > 0) est_a = est_b = 1e30;
+    // Schedule 4, never picked by the model: the pair-of-CTAs kernel, where the call has the
+    // shape it needs (head_dim 128, no sliding window, groups of a multiple of four query heads,
+    // so that pairs 2i and 2i+1 cover the same rows of one KV head).
+    const bool use2 = kv->schedule == 4 && G % 4 == 0 && c.head_dim == 128 && c.sliding_window <= 0 &&
+                      kv->max_clusters2 > 0 && kv->kernel_path == 0 && pair0 % 2 == 0;
     hdr.cluster = 0;
-    if (best_c > 0 && est_c < est_a && est_c < est_b) {
+    hdr.pair_of_ctas = 0;
+    if (!use2 && best_c > 0 && est_c < est_a && est_c < est_b) {
       // the kernel derives every CTA's part from the pair itself; no tables
       hdr.cluster = best_c;
       hdr.n_ctas = pair0 * best_c;
@@ -542,7 +552,53 @@ int run_call(pdd_kv* kv, const pdd_batch* b, const void* q, const void* k, const
     }
     const bool exact = est_b < est_a;
     const int n_ctas = exact ? n_b : n_a;
-    if (hdr.cluster == 0) {
+    if (use2) {
+      // The unit is a quad (pairs 2i and 2i+1), the shares are equal over the clusters, and CTA
+      // `rank` of cluster i takes pair 2 * quad + rank.  Scratch slots: CTA (rank, i) has index
+      // rank * n_cl + i, so the segments of a split pair lie in consecutive indices, which is
+      // what the merge kernel expects.
+      const int n_quads = pair0 / 2;
+      int64_t total_q = 0;
+      for (int i = 0; i < n_quads; ++i) total_q += nb[2 * i];
+      const int n_cl = (int)std::max<int64_t>(
+          1, std::min<int64_t>(std::min(kv->max_clusters2, kMaxAttnCtas / 2), total_q / kMinUnitsPerCta));
+      hdr.pair_of_ctas = 1;
+      hdr.n_ctas = 2 * n_cl;
+      hdr.cta_off = (int32_t)used;
+      CtaStart* cs = reinterpret_cast<CtaStart*>(rec_h + used);
+      first_unit.assign(n_cl + 1, 0);
+      for (int i = 0; i <= n_cl; ++i) first_unit[i] = total_q * i / n_cl;
+      int quad = 0;
+      int64_t quad_first = 0;
+      for (int i = 0; i <= n_cl; ++i) {
+        const int64_t u = first_unit[i];
+        while (quad < n_quads && quad_first + nb[2 * quad] <= u) quad_first += nb[2 * quad++];
+        cs[i].pair = quad;
+        cs[i].kb = (int32_t)(u - quad_first);
+      }
+      used += sizeof(CtaStart) * (size_t)(n_cl + 1);
+      hdr.split_off = (int32_t)used;
+      SplitPair* sp = reinterpret_cast<SplitPair*>(rec_h + used);
+      int n_split = 0;
+      for (int i = 1; i < n_cl; ++i) {
+        if (cs[i].kb == 0) continue;
+        if (n_split > 0 && sp[n_split - 1].pair == 2 * cs[i].pair + 1) {
+          ++sp[n_split - 2].n_seg;
+          ++sp[n_split - 1].n_seg;
+          continue;
+        }
+        const int64_t quad_start = first_unit[i] - cs[i].kb;
+        for (int rk = 0; rk < 2; ++rk) {
+          sp[n_split].pair = 2 * cs[i].pair + rk;
+          sp[n_split].cta_first = rk * n_cl + i - 1;
+          sp[n_split].n_seg = 2;
+          sp[n_split].slot_first = first_unit[i - 1] < quad_start ? 1 : 0;
+          ++n_split;
+        }
+      }
+      hdr.n_split = n_split;
+      used += sizeof(SplitPair) * (size_t)n_split;
+    } else if (hdr.cluster == 0) {
       hdr.n_ctas = n_ctas;
       hdr.cta_off = (int32_t)used;
       CtaStart* cs = reinterpret_cast<CtaStart*>(rec_h + used);
@@ -743,6 +799,7 @@ int pdd_kv_alloc(const pdd_kv_config* cfg, void* dev_buf, size_t bytes, void* st
   if (!rc) {
     // kernel attributes once per handle, not per launch
     cudaError_t pe = prepare_attn_tc(g.d, g.window != kNoWindow, kv->max_clusters);
+    if (pe == cudaSuccess && g.d == 128 && g.window == kNoWindow) pe = prepare_attn_tc2(&kv->max_clusters2);
     if (pe == cudaSuccess) pe = prepare_colsum_tc(g.d);
     if (pe == cudaSuccess)
       pe = g.d == 128 ? cudaFuncSetAttribute(attn_tc_v0_kernel<128>,
@@ -1261,7 +1318,7 @@ int pdd_set_kernel_path(pdd_kv* kv, int32_t path) {
 
 int pdd_set_schedule(pdd_kv* kv, int32_t mode) {
   if (!kv) return fail(PDD_ERR_INVALID, "null handle");
-  if (mode < 0 || mode > 3) return fail(PDD_ERR_INVALID, "mode must be 0..3");
+  if (mode < 0 || mode > 4) return fail(PDD_ERR_INVALID, "mode must be 0..4");
   kv->schedule = mode;
   return PDD_OK;
 }

@@ -268,6 +268,75 @@ __device__ __forceinline__ void mma_ts_k64(uint32_t d_tmem, uint32_t a_tmem, uin
       : "memory");
 }
 
+// ---- pair-of-CTAs (cta_group::2) forms: issued by one thread of the leader CTA for both CTAs
+__device__ __forceinline__ void tmem_alloc2(uint32_t* dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                   smem_u32(dst_smem)), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void mma2_ss_k64_first(uint32_t d_tmem, uint64_t a, uint64_t b,
+                                                  uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred pz, po;\n\t.reg .b64 a1, b1;\n\t"
+      "setp.ne.u32 pz, 0, 0;\n\tsetp.eq.u32 po, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, pz;\n\t"
+      "add.u64 a1, %1, 2;\n\tadd.u64 b1, %2, 2;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, po;\n\t"
+      "add.u64 a1, %1, 4;\n\tadd.u64 b1, %2, 4;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, po;\n\t"
+      "add.u64 a1, %1, 6;\n\tadd.u64 b1, %2, 6;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, po;\n\t}" ::"r"(d_tmem),
+      "l"(a), "l"(b), "r"(idesc)
+      : "memory");
+}
+__device__ __forceinline__ void mma2_ss_k64_acc(uint32_t d_tmem, uint64_t a, uint64_t b,
+                                                uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred po;\n\t.reg .b64 a1, b1;\n\t"
+      "setp.eq.u32 po, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, po;\n\t"
+      "add.u64 a1, %1, 2;\n\tadd.u64 b1, %2, 2;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, po;\n\t"
+      "add.u64 a1, %1, 4;\n\tadd.u64 b1, %2, 4;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, po;\n\t"
+      "add.u64 a1, %1, 6;\n\tadd.u64 b1, %2, 6;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, po;\n\t}" ::"r"(d_tmem),
+      "l"(a), "l"(b), "r"(idesc)
+      : "memory");
+}
+// O (+)= P V over 64 keys: A = P (K-major, 32 bytes per step of 16 keys), B = V rows, 2048 bytes per step
+__device__ __forceinline__ void mma2_ss_pv_k64(uint32_t d_tmem, uint64_t a, uint64_t b,
+                                               uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred pf, po;\n\t.reg .b64 a1, b1;\n\t"
+      "setp.ne.u32 pf, %4, 0;\n\tsetp.eq.u32 po, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, pf;\n\t"
+      "add.u64 a1, %1, 2;\n\tadd.u64 b1, %2, 128;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, po;\n\t"
+      "add.u64 a1, %1, 4;\n\tadd.u64 b1, %2, 256;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, po;\n\t"
+      "add.u64 a1, %1, 6;\n\tadd.u64 b1, %2, 384;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, po;\n\t}" ::"r"(d_tmem),
+      "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once all MMAs
+// issued so far by this thread have completed
+__device__ __forceinline__ void mma2_commit_both(uint64_t* bar) {
+  const uint16_t mask = 3;
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 "
+      "[%0], %1;" ::"r"(smem_u32(bar)), "h"(mask)
+      : "memory");
+}
+
 // mbarrier arrive once all previously issued MMAs of this thread have completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(

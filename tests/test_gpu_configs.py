@@ -34,10 +34,11 @@ def sampled_rows(s: wl.Sequence, n: int, seed: int) -> np.ndarray:
     return np.unique(rows)
 
 
-def run_big(w: wl.Workload):
+def run_big(w: wl.Workload, schedule: int = 0):
     """All calls through the C ABI; outputs stay on the device per call."""
     import torch
     kv = H.make_cache(w, 0)
+    kv.set_schedule(schedule)
     outs = [dict() for _ in w.seqs]          # pos0 -> device tensor
     for kind, win, group in H.batched_steps(w):
         q = np.concatenate([w.seqs[si].q[c.pos0:c.pos0 + c.length] for si, c in group])
@@ -107,12 +108,14 @@ def test_config2_full(window):
     assert int(tight.sum()) <= 64, "tight band holds %d positions" % int(tight.sum())
 
 
-def test_config4_long_prompt_sampled():
-    """Config 4 at full size (32768 + 256 tokens, 1% outlier keys x8)."""
+@pytest.mark.parametrize("schedule", [0, 4], ids=["model", "cta_pairs"])
+def test_config4_long_prompt_sampled(schedule):
+    """Config 4 at full size (32768 + 256 tokens, 1% outlier keys x8): as the cost model cuts
+    it, and through the pair-of-CTAs kernel."""
     orc = _orc()
     w = wl.config_c4("last")
     s = w.seqs[0]
-    kv, outs = run_big(w)
+    kv, outs = run_big(w, schedule)
     rows = sampled_rows(s, 48, 4)
     q64, k64, v64 = (a.astype(np.float64) for a in (s.q, s.k, s.v))
     want, _ = orc.attention_rows(q64, k64, v64, w.softmax_scale, rows)

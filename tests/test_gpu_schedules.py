@@ -1,7 +1,7 @@
 """GPU parity of each way the attention kernel's work is cut among CTAs (whole tile pairs,
 equal shares merged by a second kernel, one thread-block cluster per pair merged through
-distributed shared memory), forced one at a time on workloads the cost model would send
-elsewhere: even and odd GQA group sizes, both head dims, ragged tails, pairs with fewer key
+distributed shared memory, the pair-of-CTAs kernel where the shape allows it), forced one at
+a time on workloads the cost model would send elsewhere: even and odd GQA group sizes, both head dims, ragged tails, pairs with fewer key
 blocks than cluster CTAs, a batch of sequences, and the sliding window."""
 import dataclasses
 
@@ -13,7 +13,7 @@ from tests import helpers as H
 
 pytestmark = pytest.mark.gpu
 
-MODES = [1, 2, 3]
+MODES = [1, 2, 3, 4]
 
 CASES = [
     # name, seed, hq, hkv, d, n_prompt, chunk, n_received, page, obs. window, sliding window
@@ -24,6 +24,8 @@ CASES = [
     ("few_pairs_long", 704, 2, 1, 128, 2300, 256, 40, 64, "last", 0),
     ("band_g4", 705, 8, 2, 128, 1500, 512, 9, 64, "all", 300),
     ("band_rowpairs", 706, 3, 3, 128, 1400, 700, 3, 64, "all", 200),
+    ("g8_long_d128", 707, 16, 2, 128, 3000, 1024, 40, 64, "last", 0),
+    ("g4_ragged_tail", 708, 4, 1, 128, 1333, 777, 21, 128, "all", 0),
 ]
 
 
@@ -52,10 +54,10 @@ def test_forced_schedule_ragged_batch(mode):
 
 
 def test_schedules_agree_with_each_other():
-    """Same inputs, three cuts: outputs differ only by the rounding order of the merge."""
+    """Same inputs, four cuts: outputs differ only by the rounding order of the merge."""
     w = wl.small_like("sched_agree", 710, 8, 2, 128, 1200, 400, 16, window="all")
     res = []
-    for mode in (1, 2, 3):
+    for mode in (1, 2, 3, 4):
         kv = H.make_cache(w, 0)
         kv.set_schedule(mode)
         res.append(H.run_library(w, cache=kv)[0])
@@ -70,6 +72,6 @@ def test_bad_schedule_mode_is_rejected():
     w = wl.small_like("sched_bad", 711, 2, 2, 64, 10, 10, 0)
     kv = H.make_cache(w, 0)
     with pytest.raises(B.PddError) as e:
-        kv.set_schedule(4)
+        kv.set_schedule(5)
     assert e.value.status == B.PDD_ERR_INVALID
     kv.close()
